@@ -1,0 +1,170 @@
+/*
+ * libmoe — top-2 Mixture-of-Experts layer forward with expert pruning and
+ * dynamic expert skipping, and the layer-wise pruning search
+ * (arXiv 2402.14800), as CUDA kernels for sm_100a.
+ *
+ * C ABI.  Conventions shared by every call:
+ *   - "device" pointers are CUDA device memory of the current device, owned by
+ *     the caller unless stated; "host" pointers are ordinary host memory.
+ *   - bf16 tensors are row-major with the last index contiguous and a 16-byte
+ *     aligned base address.
+ *   - Calls return MOE_OK (0) or a negative moe_status; moe_layer_create returns
+ *     NULL on failure.  moe_last_error() gives a thread-local message for the
+ *     last failing call.  No C++ exception crosses this boundary.
+ *   - Work is enqueued on the handle's stream (default: the legacy stream 0) and
+ *     is asynchronous unless the call returns results to host memory.
+ *   - A handle must not be used from two host threads at once: its scratch
+ *     buffers are shared by all of its calls.
+ */
+#ifndef MOE_H_
+#define MOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum moe_status {
+  MOE_OK = 0,
+  MOE_ERR_INVALID_ARG = -1,       /* null/misaligned pointer, bad mask, r out of range, ... */
+  MOE_ERR_UNSUPPORTED_SHAPE = -2, /* h or f not a multiple of 64, E > 16, ... */
+  MOE_ERR_CUDA = -3,              /* a CUDA runtime/driver call failed */
+  MOE_ERR_OOM = -4,               /* device memory for weights or scratch not available */
+  MOE_ERR_DEVICE_TIMEOUT = -5,    /* a bounded wait inside a kernel expired */
+  MOE_ERR_ARCH = -6               /* the current device is not sm_100 */
+} moe_status;
+
+#define MOE_MAX_EXPERTS 16
+
+typedef struct moe_layer moe_layer_t; /* opaque, owned by the library */
+
+/*
+ * Build one MoE layer (Sec. 3.1) restricted to the kept experts (Sec. 3.2:
+ * pruned experts are discarded together with their router rows).
+ *   W_gate [E][h]     bf16 device   router, one row per expert
+ *   W1     [E][f][h]  bf16 device   gate projection of the SwiGLU expert
+ *   W3     [E][f][h]  bf16 device   up projection
+ *   W2     [E][h][f]  bf16 device   down projection
+ *   kept_mask         bit e set <=> expert e is kept; at least 2 bits (top-2)
+ * The kept router rows and kept experts are COPIED into library-owned buffers
+ * in the layout the kernels want, so the handle occupies popcount(mask)/E of
+ * the layer's bytes and the caller may free its tensors when this returns
+ * (the call synchronises the device).  Requires h % 64 == 0, f % 64 == 0,
+ * 2 <= E <= 16, and an sm_100 device.
+ */
+moe_layer_t* moe_layer_create(const void* W_gate, const void* W1, const void* W3, const void* W2,
+                              int h, int f, int E, uint32_t kept_mask);
+
+/* Free the handle with its weights and scratch (synchronises its stream). */
+void moe_layer_destroy(moe_layer_t* layer);
+
+/* Stream (a cudaStream_t) that later calls on this handle enqueue on. */
+int moe_set_stream(moe_layer_t* layer, void* cuda_stream);
+
+/* Bytes of device memory the handle holds for weights (router + kept experts). */
+size_t moe_layer_weight_bytes(const moe_layer_t* layer);
+
+/* Bytes of device memory the handle currently holds as scratch. */
+size_t moe_layer_scratch_bytes(const moe_layer_t* layer);
+
+/*
+ * Layer forward for T tokens (Sec. 3.1 Eq. 1-2, Sec. 3.2, Sec. 3.3, App. A.2):
+ *   l = W_gate x over the kept experts, w = Softmax(l), e0/e1 = top-2 (ties to
+ *   the lower expert index), e1 is skipped when w_e1 < beta * w_e0 (strict),
+ *   z = w~_e0 E_e0(x) + w~_e1 E_e1(x) with w~ renormalised over the experts
+ *   that run (w~_e0 = 1 after a skip), E_e(x) = W2_e (silu(W1_e x) * W3_e x).
+ *   The SwiGLU activation and y are rounded to bf16; everything else is fp32.
+ *   x [T][h] bf16 device (read), y [T][h] bf16 device (written); beta >= 0,
+ *   beta = 0 never skips.  x and y may not overlap.  T = 0 is a no-op.
+ *   routing_stats: NULL, or device memory of moe_routing_stats_bytes(T, E)
+ *   bytes that receives the per-token routing record (layout below).
+ * Asynchronous; nothing is retained after the kernels finish.
+ */
+int moe_forward(moe_layer_t* layer, const void* x, int T, float beta, void* y,
+                void* routing_stats);
+
+/* As moe_forward, but y = bf16(residual + z) with one rounding.  residual
+ * [T][h] bf16 device may be the same buffer as y; NULL means 0. */
+int moe_forward_residual(moe_layer_t* layer, const void* x, int T, float beta,
+                         const void* residual, void* y, void* routing_stats);
+
+/*
+ * moe_forward with HOST buffers: copies x_host to the device, runs the layer,
+ * copies y back and waits for it.  x_host/y_host [T][h] bf16; pinned memory
+ * makes the copies asynchronous to the host but is not required.
+ */
+int moe_forward_host(moe_layer_t* layer, const void* x_host, int T, float beta, void* y_host);
+
+/*
+ * Routing record written by moe_forward when routing_stats != NULL.  Sections
+ * in this order, each starting at a multiple of 16 bytes:
+ *   int32  idx[T][2]      original ids of e0, e1
+ *   float  wn[T][2]       weights applied to E_e0, E_e1 (1, 0 after a skip)
+ *   float  ratio[T]       w_e1 / w_e0
+ *   uint8  skipped[T]
+ *   int32  count[E][2]    token-expert pairs that ran, per expert and slot
+ *   int32  n_skipped
+ *   int32  n_experts_touched   experts with at least one pair
+ * moe_routing_stats_layout fills offsets[7] (bytes from the start, same order)
+ * and returns the total size; moe_routing_stats_bytes returns only the size.
+ */
+size_t moe_routing_stats_layout(int T, int E, size_t offsets[7]);
+size_t moe_routing_stats_bytes(int T, int E);
+
+/*
+ * beta for dynamic skipping (Sec. 3.3): the median over the T calibration
+ * tokens of w_e1 / w_e0 under this layer's router; for even T the mean of the
+ * two middle values.  x [T][h] bf16 device, T >= 1; *beta_out is host memory.
+ * Synchronises the handle's stream.
+ */
+int moe_calibrate_beta(moe_layer_t* layer, const void* x, int T, float* beta_out);
+
+/*
+ * Layer-wise expert pruning search (Sec. 3.2, Eq. 3).  For every subset C of r
+ * experts, in lexicographic order of the ascending index tuples, the pruned
+ * layer F'(x, C) (router rows of the other experts removed, no skipping) is
+ * compared with the unpruned layer F(x) over the T calibration tokens:
+ *   losses[i] = || F'(x, C_i) - F(x) ||_F        (host, C(E, r) floats)
+ *   *best_subset = bitmask of the first subset with the smallest loss (host)
+ * Every expert is evaluated once per token (outputs kept in bf16) and each
+ * subset only re-routes among its kept logits and gathers.  The handle must
+ * have been created with all E experts kept; 2 <= r <= E.  x_calib [T][h] bf16
+ * device, T >= 1.  Synchronises the handle's stream.
+ */
+int moe_prune_search(moe_layer_t* layer, const void* x_calib, int T, int r, float* losses,
+                     uint32_t* best_subset);
+
+/* Number of subsets moe_prune_search scores: C(E, r), 0 if out of range. */
+long moe_num_subsets(int E, int r);
+
+/*
+ * RMSNorm with unit gain, out = bf16(x / sqrt(mean(x^2) + eps)), the
+ * normalisation placed before each MoE layer when layers are stacked.
+ * x, out [T][h] bf16 device (may alias); stream is a cudaStream_t.
+ */
+int moe_rmsnorm(const void* x, int T, int h, float eps, void* out, void* cuda_stream);
+
+/*
+ * A stack of MoE layers with attention left out:
+ *   x_{l+1} = x_l + MoE_l(RMSNorm(x_l)),  l = 0 .. n_layers-1,
+ * each layer with its own kept experts and its own betas[l] (host array, NULL
+ * for no skipping).  x [T][h] bf16 device is not modified; y [T][h] receives
+ * x_{n_layers}.  All layers must share h and run on the first layer's stream.
+ * eps is the RMSNorm epsilon.
+ */
+int moe_stack_forward(moe_layer_t* const* layers, int n_layers, const void* x, int T,
+                      const float* betas, float eps, void* y);
+
+/* 0 when no kernel of this handle has reported a bounded wait expiring since
+ * the last call of this function, else MOE_ERR_DEVICE_TIMEOUT.  Synchronises. */
+int moe_device_status(moe_layer_t* layer);
+
+/* Message of the last failing call on this host thread ("" if none). */
+const char* moe_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_H_ */

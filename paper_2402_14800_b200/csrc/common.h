@@ -1,0 +1,126 @@
+// Internal declarations shared by the translation units of libmoe.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "moe.h"
+
+namespace moe {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kMaxE = MOE_MAX_EXPERTS;
+constexpr int kTileRows = 128;            // token rows per row tile of the grouped GEMMs
+constexpr int kRouteTokPerBlock = 64;     // tokens routed by one block (8 warps x 8 tokens)
+constexpr int kHistCols = 2 * kMaxE + 1;  // per (expert, slot) pair counts + skipped count
+constexpr int kInterleave = 16;           // W1/W3 rows are interleaved in groups of 16
+constexpr int kDecodeMaxT = 256;          // up to here the weight-stationary GEMM is used
+constexpr int kDecodeKbPerItem = 32;      // k-blocks (of 64) per split-K item, decode down-proj
+
+// Device-resident description of one permuted batch, written by the scan kernel
+// (or by set_dense_meta for the search) and read by every later kernel.
+struct Meta {
+  int32_t count[kMaxE];            // token-expert pairs that run, per kept expert (compact index)
+  int32_t count_slot[kMaxE][2];    // the same, split by top-2 slot
+  int32_t off[kMaxE + 1];          // first permuted row of each expert's group (padded groups)
+  int32_t tile_prefix[kMaxE + 1];  // cumulative number of 128-row tiles
+  int32_t rows_total;              // off[r]
+  int32_t n_skipped;
+  int32_t n_touched;
+  int32_t reserved;
+};
+
+struct KeptIds {
+  int32_t id[kMaxE];  // compact index -> original expert id
+};
+
+// ---- routing / permutation / element-wise kernels (route_permute.cu) --------------------
+struct RouteOut {
+  int32_t* idx;       // [T][2] compact expert index
+  float* wn;          // [T][2]
+  float* ratio;       // [T]
+  uint8_t* skipped;   // [T]
+  float* logits;      // [T][r] or null
+  int32_t* blk_hist;  // [nblk][kHistCols] or null
+  // user-visible routing record (all null when not requested)
+  int32_t* s_idx;
+  float* s_wn;
+  float* s_ratio;
+  uint8_t* s_skipped;
+};
+
+cudaError_t launch_router(const bf16* x, const bf16* Wg, int T, int h, int r, float beta,
+                          const KeptIds& kept, const RouteOut& out, cudaStream_t st);
+cudaError_t launch_scan(const int32_t* blk_hist, int nblk, int r, int pad, int32_t* blk_base,
+                        Meta* meta, int32_t* s_count, int32_t* s_nskipped, int32_t* s_ntouched,
+                        const KeptIds& kept, int E, cudaStream_t st);
+cudaError_t launch_scatter(const int32_t* idx, const uint8_t* skipped, const int32_t* blk_base,
+                           const Meta* meta, int T, int32_t* pair_pos, int32_t* row_token,
+                           cudaStream_t st);
+cudaError_t launch_gather(const bf16* x, const int32_t* row_token, const Meta* meta, int h,
+                          int cap_rows, bf16* xperm, cudaStream_t st);
+cudaError_t launch_combine(const float* O, int ksplit, size_t split_stride, const int32_t* pair_pos,
+                           const float* wn, const bf16* residual, int T, int h, bf16* y,
+                           cudaStream_t st);
+cudaError_t launch_rmsnorm(const bf16* x, int T, int h, float eps, bf16* out, cudaStream_t st);
+cudaError_t launch_set_dense_meta(Meta* meta, int E, int rows_per_expert, int off_stride,
+                                  cudaStream_t st);
+// k-th smallest (0-based) of ratio[T] for k = k0 and k1, written to out[0], out[1]
+cudaError_t launch_select2(const float* ratio, int T, int k0, int k1, float* out, cudaStream_t st);
+// W13[c][32q + s] = W1[id[c]][16q + s] (s < 16) | W3[id[c]][16q + s - 16] (s >= 16)
+cudaError_t launch_interleave(const bf16* W1, const bf16* W3, const KeptIds& kept, int r, int f,
+                              int h, bf16* W13, cudaStream_t st);
+
+// ---- grouped GEMMs (gemm_sm100.cu) ----------------------------------------------------
+enum GemmOut { kOutActBf16 = 0, kOutF32 = 1, kOutBf16 = 2 };
+
+struct GemmArgs {
+  const Meta* meta;
+  int r;         // kept experts
+  int K;         // contraction length (h for gate/up, f for down)
+  int n_w_rows;  // weight rows per expert (2f interleaved for gate/up, h for down)
+  // token-side operand rows: a_row = a_row_base + a_off_mul * off[c] + 128 * m
+  int a_row_base, a_off_mul;
+  // output rows: out_row = out_row_base + out_off_mul * off[c] + 128 * m; column offset c * out_col_mul
+  int out_row_base, out_off_mul;
+  long long out_col_mul;
+  long long out_ld;        // elements between output rows
+  void* out;               // bf16 activations / fp32 outputs / bf16 expert outputs
+  long long split_stride;  // elements between split-K partial planes (decode down-proj)
+  int* status;             // device error word
+};
+
+int gemm_init_driver_api();  // resolves cuTensorMapEncodeTiled; 0 on success
+int make_map_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows);
+int make_map_3d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows, uint64_t planes,
+                uint32_t box_rows);
+
+struct GemmMaps {
+  CUtensorMap w;     // weights [planes = r][rows][K], box 64 x (256 or 128) x 1
+  CUtensorMap t[4];  // token-side operand [rows][K], boxes of 16 / 32 / 64 / 128 rows
+};
+
+// Token rows are the 128-row MMA operand, weights the 256-wide one (large T).
+cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps& maps,
+                                 const GemmArgs& a, cudaStream_t st);
+// Weight rows are the 128-row MMA operand, tokens the narrow one (small T): weights stream once.
+cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
+                                  int kb_per_item, cudaStream_t st);
+// Plain CUDA-core kernels of the same contractions, for bring-up and debugging only
+// (MOE_DEBUG_SIMT=1); never selected otherwise.
+cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,
+                                cudaStream_t st);
+cudaError_t launch_simt_down(const bf16* A, const bf16* W2, const GemmArgs& a, int cap_rows,
+                             GemmOut out_kind, cudaStream_t st);
+cudaError_t gemm_set_attributes();
+
+// ---- search (search.cu) ---------------------------------------------------------------
+int enumerate_num_blocks(int T);
+cudaError_t launch_enumerate(const float* logits, const bf16* Yall, int T, int E, int r, int h,
+                             const uint32_t* subsets, int nC, float* partial, double* loss_sq,
+                             float* losses, cudaStream_t st);
+
+}  // namespace moe

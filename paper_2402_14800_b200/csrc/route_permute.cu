@@ -1,0 +1,485 @@
+// Router, token permutation, combine and the small element-wise kernels.
+//
+//   router_kernel   Sec. 3.1 (logits, softmax, top-2, Eq. 1), Sec. 3.2 (kept experts only),
+//                   Sec. 3.3 (skip test), App. A.2 (weight 1 after a skip); warp per token.
+//   scan / scatter  stable counting sort of the token-expert pairs that run, by expert;
+//                   no atomics, the order is a function of the routing alone.
+//   gather          copies the routed rows of x into expert-contiguous order.
+//   combine         Eq. 2: y = bf16(residual + w~_e0 o_e0 + w~_e1 o_e1), slot 0 first.
+#include "common.h"
+
+namespace moe {
+
+namespace {
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+  f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x);
+  f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
+  f[4] = bf16_lo(v.z); f[5] = bf16_hi(v.z);
+  f[6] = bf16_lo(v.w); f[7] = bf16_hi(v.w);
+}
+
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+// ------------------------------------------------------------------------------- router
+
+template <int R>
+__global__ void __launch_bounds__(256)
+router_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, int h, int r,
+              float beta, KeptIds kept, RouteOut o) {
+  __shared__ int s_e[kRouteTokPerBlock][2];
+  __shared__ int s_skip[kRouteTokPerBlock];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t0 = blockIdx.x * kRouteTokPerBlock;
+  const int nvec = h >> 3;
+
+  for (int i = 0; i < kRouteTokPerBlock / 8; ++i) {
+    const int tl = warp * (kRouteTokPerBlock / 8) + i;
+    const int t = t0 + tl;
+    if (t >= T) {
+      if (lane == 0) { s_e[tl][0] = -1; s_e[tl][1] = -1; s_skip[tl] = 0; }
+      continue;
+    }
+    float acc[R];
+#pragma unroll
+    for (int c = 0; c < R; ++c) acc[c] = 0.f;
+    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)t * h);
+    for (int v = lane; v < nvec; v += 32) {
+      float xf[8];
+      unpack8(__ldg(xr + v), xf);
+#pragma unroll
+      for (int c = 0; c < R; ++c) {
+        if (c < r) {
+          float wf[8];
+          unpack8(__ldg(reinterpret_cast<const uint4*>(Wg + (size_t)c * h) + v), wf);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) acc[c] = fmaf(xf[k], wf[k], acc[c]);
+        }
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < R; ++c) {
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], s);
+    }
+    if (lane == 0) {
+      // top-2 on the logits (softmax is increasing), ties to the lower index
+      int e0 = 0;
+      float l0 = acc[0];
+#pragma unroll
+      for (int c = 1; c < R; ++c)
+        if (c < r && acc[c] > l0) { l0 = acc[c]; e0 = c; }
+      int e1 = -1;
+      float l1 = 0.f;
+#pragma unroll
+      for (int c = 0; c < R; ++c)
+        if (c < r && c != e0 && (e1 < 0 || acc[c] > l1)) { l1 = acc[c]; e1 = c; }
+      // softmax numerators relative to the maximum: p_e0 = 1, p_e1 = exp(l1 - l0); the
+      // denominator cancels in the ratio, the skip test and the normalised weights
+      const float p1 = expf(l1 - l0);
+      const bool skip = p1 < beta * 1.0f;
+      float w0, w1;
+      if (skip) { w0 = 1.f; w1 = 0.f; }
+      else { const float d = 1.0f + p1; w0 = 1.0f / d; w1 = p1 / d; }
+      o.idx[2 * t] = e0; o.idx[2 * t + 1] = e1;
+      o.wn[2 * t] = w0; o.wn[2 * t + 1] = w1;
+      o.ratio[t] = p1;
+      o.skipped[t] = skip ? 1 : 0;
+      if (o.s_idx) {
+        o.s_idx[2 * t] = kept.id[e0]; o.s_idx[2 * t + 1] = kept.id[e1];
+        o.s_wn[2 * t] = w0; o.s_wn[2 * t + 1] = w1;
+        o.s_ratio[t] = p1;
+        o.s_skipped[t] = skip ? 1 : 0;
+      }
+      if (o.logits) {
+#pragma unroll
+        for (int c = 0; c < R; ++c)
+          if (c < r) o.logits[(size_t)t * r + c] = acc[c];
+      }
+      s_e[tl][0] = e0;
+      s_e[tl][1] = skip ? -1 : e1;
+      s_skip[tl] = skip ? 1 : 0;
+    }
+  }
+  __syncthreads();
+  if (o.blk_hist && threadIdx.x < kHistCols) {
+    int n = 0;
+    if (threadIdx.x == 2 * kMaxE) {
+      for (int i = 0; i < kRouteTokPerBlock; ++i) n += s_skip[i];
+    } else {
+      const int c = threadIdx.x >> 1, slot = threadIdx.x & 1;
+      for (int i = 0; i < kRouteTokPerBlock; ++i) n += (s_e[i][slot] == c);
+    }
+    o.blk_hist[(size_t)blockIdx.x * kHistCols + threadIdx.x] = n;
+  }
+}
+
+// ---------------------------------------------------------------------------------- scan
+
+// One block.  Warp c scans the per-block counts of expert c over the blocks in order, which
+// gives every block its first position inside the expert's group; thread 0 then lays the
+// groups out (each padded to `pad` rows) and counts the 128-row tiles.
+__global__ void __launch_bounds__(1024)
+scan_kernel(const int32_t* __restrict__ blk_hist, int nblk, int r, int pad,
+            int32_t* __restrict__ blk_base, Meta* meta, int32_t* s_count, int32_t* s_nskipped,
+            int32_t* s_ntouched, KeptIds kept, int E) {
+  __shared__ int s_tot[kMaxE][2];
+  __shared__ int s_skipped;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp < r) {
+    int run = 0, run0 = 0;
+    for (int b0 = 0; b0 < nblk; b0 += 32) {
+      const int b = b0 + lane;
+      int v0 = 0, v1 = 0;
+      if (b < nblk) {
+        v0 = blk_hist[(size_t)b * kHistCols + 2 * warp];
+        v1 = blk_hist[(size_t)b * kHistCols + 2 * warp + 1];
+      }
+      const int v = v0 + v1;
+      int inc = v;
+#pragma unroll
+      for (int s = 1; s < 32; s <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, inc, s);
+        if (lane >= s) inc += n;
+      }
+      if (b < nblk) blk_base[(size_t)b * kMaxE + warp] = run + inc - v;
+      run += __shfl_sync(0xffffffffu, inc, 31);
+      int t0 = v0;
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) t0 += __shfl_xor_sync(0xffffffffu, t0, s);
+      run0 += t0;
+    }
+    if (lane == 0) { s_tot[warp][0] = run0; s_tot[warp][1] = run - run0; }
+  } else if (warp == kMaxE) {
+    int n = 0;
+    for (int b = lane; b < nblk; b += 32) n += blk_hist[(size_t)b * kHistCols + 2 * kMaxE];
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(0xffffffffu, n, s);
+    if (lane == 0) s_skipped = n;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int off = 0, tiles = 0, touched = 0;
+    meta->off[0] = 0;
+    meta->tile_prefix[0] = 0;
+    for (int c = 0; c < kMaxE; ++c) {
+      const int n0 = c < r ? s_tot[c][0] : 0, n1 = c < r ? s_tot[c][1] : 0;
+      const int n = n0 + n1;
+      meta->count[c] = n;
+      meta->count_slot[c][0] = n0;
+      meta->count_slot[c][1] = n1;
+      off += (n + pad - 1) / pad * pad;
+      tiles += (n + kTileRows - 1) / kTileRows;
+      touched += (n > 0);
+      meta->off[c + 1] = off;
+      meta->tile_prefix[c + 1] = tiles;
+    }
+    meta->rows_total = off;
+    meta->n_skipped = s_skipped;
+    meta->n_touched = touched;
+    meta->reserved = 0;
+    if (s_count) {
+      for (int e = 0; e < E; ++e) { s_count[2 * e] = 0; s_count[2 * e + 1] = 0; }
+      for (int c = 0; c < r; ++c) {
+        s_count[2 * kept.id[c]] = s_tot[c][0];
+        s_count[2 * kept.id[c] + 1] = s_tot[c][1];
+      }
+      *s_nskipped = s_skipped;
+      *s_ntouched = touched;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------- scatter
+
+// Position of pair (t, slot) = start of its expert's group + pairs of that expert in earlier
+// blocks + pairs of that expert among the earlier tokens of this block.
+__global__ void __launch_bounds__(2 * kRouteTokPerBlock)
+scatter_kernel(const int32_t* __restrict__ idx, const uint8_t* __restrict__ skipped,
+               const int32_t* __restrict__ blk_base, const Meta* __restrict__ meta, int T,
+               int32_t* __restrict__ pair_pos, int32_t* __restrict__ row_token) {
+  __shared__ int s_e[kRouteTokPerBlock][2];
+  const int tl = threadIdx.x >> 1, slot = threadIdx.x & 1;
+  const int t = blockIdx.x * kRouteTokPerBlock + tl;
+  int c = -1;
+  if (t < T) {
+    c = idx[2 * t + slot];
+    if (slot == 1 && skipped[t]) c = -1;
+  }
+  s_e[tl][slot] = c;
+  __syncthreads();
+  if (t >= T) return;
+  int pos = -1;
+  if (c >= 0) {
+    int rank = 0;
+    for (int i = 0; i < tl; ++i) rank += (s_e[i][0] == c) + (s_e[i][1] == c);
+    pos = meta->off[c] + blk_base[(size_t)blockIdx.x * kMaxE + c] + rank;
+    row_token[pos] = t;
+  }
+  pair_pos[2 * t + slot] = pos;
+}
+
+// -------------------------------------------------------------------------------- gather
+
+__global__ void __launch_bounds__(256)
+gather_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ row_token,
+              const Meta* __restrict__ meta, int h, bf16* __restrict__ xperm) {
+  const int rows = meta->rows_total;
+  const int lane = threadIdx.x & 31;
+  const int nvec = h >> 3;
+  for (int row = blockIdx.x * 8 + (threadIdx.x >> 5); row < rows; row += gridDim.x * 8) {
+    const int t = row_token[row];
+    uint4* dst = reinterpret_cast<uint4*>(xperm + (size_t)row * h);
+    if (t >= 0) {
+      const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * h);
+      for (int v = lane; v < nvec; v += 32) dst[v] = __ldg(src + v);
+    } else {
+      for (int v = lane; v < nvec; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------- combine
+
+__global__ void __launch_bounds__(128)
+combine_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
+               const int32_t* __restrict__ pair_pos, const float* __restrict__ wn,
+               const bf16* residual, int T, int h, bf16* y) {
+  const int t = blockIdx.x;
+  const int p0 = pair_pos[2 * t], p1 = pair_pos[2 * t + 1];
+  const float w0 = wn[2 * t], w1 = wn[2 * t + 1];
+  const int nvec = h >> 3;
+  for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+    float a[8], b[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { a[k] = 0.f; b[k] = 0.f; }
+    for (int s = 0; s < ksplit; ++s) {
+      const float4* o0 = reinterpret_cast<const float4*>(O + s * split_stride + (size_t)p0 * h) + 2 * v;
+      const float4 q0 = o0[0], q1 = o0[1];
+      a[0] += q0.x; a[1] += q0.y; a[2] += q0.z; a[3] += q0.w;
+      a[4] += q1.x; a[5] += q1.y; a[6] += q1.z; a[7] += q1.w;
+      if (p1 >= 0) {
+        const float4* o1 = reinterpret_cast<const float4*>(O + s * split_stride + (size_t)p1 * h) + 2 * v;
+        const float4 r0 = o1[0], r1 = o1[1];
+        b[0] += r0.x; b[1] += r0.y; b[2] += r0.z; b[3] += r0.w;
+        b[4] += r1.x; b[5] += r1.y; b[6] += r1.z; b[7] += r1.w;
+      }
+    }
+    float z[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) z[k] = (p1 >= 0) ? fmaf(w1, b[k], w0 * a[k]) : w0 * a[k];
+    if (residual) {
+      float rf[8];
+      unpack8(reinterpret_cast<const uint4*>(residual + (size_t)t * h)[v], rf);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) z[k] += rf[k];
+    }
+    uint4 outv;
+    outv.x = pack2(z[0], z[1]); outv.y = pack2(z[2], z[3]);
+    outv.z = pack2(z[4], z[5]); outv.w = pack2(z[6], z[7]);
+    reinterpret_cast<uint4*>(y + (size_t)t * h)[v] = outv;
+  }
+}
+
+// ------------------------------------------------------------------------------- rmsnorm
+
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(const bf16* x, int T, int h, float eps, bf16* out) {
+  __shared__ float s_part[8];
+  const int t = blockIdx.x;
+  const int nvec = h >> 3;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)t * h);
+  float ss = 0.f;
+  for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+    float f[8];
+    unpack8(xr[v], f);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) ss = fmaf(f[k], f[k], ss);
+  }
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, s);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += s_part[w];
+  const float inv = 1.0f / sqrtf(tot / (float)h + eps);
+  for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+    float f[8];
+    unpack8(xr[v], f);
+    uint4 o;
+    o.x = pack2(f[0] * inv, f[1] * inv); o.y = pack2(f[2] * inv, f[3] * inv);
+    o.z = pack2(f[4] * inv, f[5] * inv); o.w = pack2(f[6] * inv, f[7] * inv);
+    reinterpret_cast<uint4*>(out + (size_t)t * h)[v] = o;
+  }
+}
+
+// ---------------------------------------------------------------------------- dense meta
+
+__global__ void set_dense_meta_kernel(Meta* meta, int E, int rows, int off_stride) {
+  if (threadIdx.x != 0) return;
+  const int tiles = (rows + kTileRows - 1) / kTileRows;
+  for (int c = 0; c <= kMaxE; ++c) {
+    const int cc = c < E ? c : E;
+    meta->off[c] = cc * off_stride;
+    meta->tile_prefix[c] = cc * tiles;
+    if (c < kMaxE) {
+      meta->count[c] = c < E ? rows : 0;
+      meta->count_slot[c][0] = meta->count[c];
+      meta->count_slot[c][1] = 0;
+    }
+  }
+  meta->rows_total = E * off_stride;
+  meta->n_skipped = 0;
+  meta->n_touched = E;
+  meta->reserved = 0;
+}
+
+// -------------------------------------------------------------------------------- select
+
+__device__ __forceinline__ uint32_t float_key(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// Exact k-th smallest by radix selection on the ordered bit patterns, 8 bits per pass.
+__global__ void __launch_bounds__(1024)
+select2_kernel(const float* __restrict__ v, int n, int k0, int k1, float* out) {
+  __shared__ unsigned hist[256];
+  __shared__ unsigned s_prefix;
+  __shared__ int s_k;
+  for (int which = 0; which < 2; ++which) {
+    if (threadIdx.x == 0) { s_prefix = 0; s_k = which ? k1 : k0; }
+    unsigned mask = 0;
+    for (int pass = 3; pass >= 0; --pass) {
+      const int shift = pass * 8;
+      if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+      __syncthreads();
+      const unsigned prefix = s_prefix;
+      for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const unsigned key = float_key(v[i]);
+        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        int k = s_k;
+        unsigned bin = 0;
+        for (; bin < 255; ++bin) {
+          if (k < (int)hist[bin]) break;
+          k -= (int)hist[bin];
+        }
+        s_k = k;
+        s_prefix = prefix | (bin << shift);
+      }
+      mask |= 0xffu << shift;
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) out[which] = key_float(s_prefix);
+    __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------------------- interleave
+
+__global__ void __launch_bounds__(256)
+interleave_kernel(const bf16* __restrict__ W1, const bf16* __restrict__ W3, KeptIds kept, int r,
+                  int f, int h, bf16* __restrict__ W13) {
+  const long long rows = (long long)r * 2 * f;
+  const int lane = threadIdx.x & 31;
+  const int nvec = h >> 3;
+  for (long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5); row < rows;
+       row += (long long)gridDim.x * 8) {
+    const int c = (int)(row / (2 * f));
+    const int R = (int)(row % (2 * f));
+    const int q = R / (2 * kInterleave), s = R % (2 * kInterleave);
+    const bf16* src = (s < kInterleave)
+        ? W1 + ((size_t)kept.id[c] * f + (size_t)q * kInterleave + s) * h
+        : W3 + ((size_t)kept.id[c] * f + (size_t)q * kInterleave + s - kInterleave) * h;
+    const uint4* sv = reinterpret_cast<const uint4*>(src);
+    uint4* dv = reinterpret_cast<uint4*>(W13 + (size_t)row * h);
+    for (int v = lane; v < nvec; v += 32) dv[v] = __ldg(sv + v);
+  }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------ launchers
+
+cudaError_t launch_router(const bf16* x, const bf16* Wg, int T, int h, int r, float beta,
+                          const KeptIds& kept, const RouteOut& out, cudaStream_t st) {
+  const int nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
+  switch (r) {
+    case 2: router_kernel<2><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+    case 3: case 4: router_kernel<4><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+    case 5: case 6: router_kernel<6><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+    case 7: case 8: router_kernel<8><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+    default: router_kernel<kMaxE><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scan(const int32_t* blk_hist, int nblk, int r, int pad, int32_t* blk_base,
+                        Meta* meta, int32_t* s_count, int32_t* s_nskipped, int32_t* s_ntouched,
+                        const KeptIds& kept, int E, cudaStream_t st) {
+  scan_kernel<<<1, 1024, 0, st>>>(blk_hist, nblk, r, pad, blk_base, meta, s_count, s_nskipped,
+                                  s_ntouched, kept, E);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scatter(const int32_t* idx, const uint8_t* skipped, const int32_t* blk_base,
+                           const Meta* meta, int T, int32_t* pair_pos, int32_t* row_token,
+                           cudaStream_t st) {
+  const int nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
+  scatter_kernel<<<nblk, 2 * kRouteTokPerBlock, 0, st>>>(idx, skipped, blk_base, meta, T, pair_pos,
+                                                         row_token);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather(const bf16* x, const int32_t* row_token, const Meta* meta, int h,
+                          int cap_rows, bf16* xperm, cudaStream_t st) {
+  int blocks = (cap_rows + 7) / 8;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  gather_kernel<<<blocks, 256, 0, st>>>(x, row_token, meta, h, xperm);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const float* O, int ksplit, size_t split_stride, const int32_t* pair_pos,
+                           const float* wn, const bf16* residual, int T, int h, bf16* y,
+                           cudaStream_t st) {
+  combine_kernel<<<T, 128, 0, st>>>(O, ksplit, split_stride, pair_pos, wn, residual, T, h, y);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rmsnorm(const bf16* x, int T, int h, float eps, bf16* out, cudaStream_t st) {
+  rmsnorm_kernel<<<T, 256, 0, st>>>(x, T, h, eps, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_set_dense_meta(Meta* meta, int E, int rows_per_expert, int off_stride,
+                                  cudaStream_t st) {
+  set_dense_meta_kernel<<<1, 32, 0, st>>>(meta, E, rows_per_expert, off_stride);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select2(const float* ratio, int T, int k0, int k1, float* out, cudaStream_t st) {
+  select2_kernel<<<1, 1024, 0, st>>>(ratio, T, k0, k1, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_interleave(const bf16* W1, const bf16* W3, const KeptIds& kept, int r, int f,
+                              int h, bf16* W13, cudaStream_t st) {
+  interleave_kernel<<<148 * 8, 256, 0, st>>>(W1, W3, kept, r, f, h, W13);
+  return cudaGetLastError();
+}
+
+}  // namespace moe
