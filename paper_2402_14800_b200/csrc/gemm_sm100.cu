@@ -1,0 +1,760 @@
+// Grouped GEMMs of the SwiGLU experts on the 5th-generation tensor cores (tcgen05),
+// operands staged in shared memory by TMA, accumulators in tensor memory.
+//
+//   E_e(x) = W2_e ( silu(W1_e x) * (W3_e x) )      (Sec. 3.1; Mixtral's SwiGLU form)
+//
+// Two persistent, warp-specialised kernels share one pipeline skeleton:
+//   gemm_tokens_m   128 token rows x 256 weight rows per tile; for large batches, where the
+//                   work is a dense contraction bound by the tensor pipe.
+//   gemm_weights_m  128 weight rows x (16..128) tokens per item; for small batches, where
+//                   every weight byte is streamed from HBM exactly once.
+// Warp 0 issues TMA loads, warp 1 issues the MMAs (one lane) and owns the tensor memory,
+// warps 2-5 run the epilogue out of tensor memory while the next tile accumulates in the
+// other half of it.
+//
+// W1/W3 are stored interleaved (16 gate rows, 16 up rows, ...) so that one accumulator tile
+// holds both halves of a SwiGLU feature and the epilogue can fuse silu(g) * u.
+//
+// Every wait on an mbarrier is bounded: when it expires the CTA raises its abort flag, all
+// roles leave their loops, outstanding copies and MMAs are drained (again bounded), tensor
+// memory is released and the device status word is set.
+#include <stdio.h>
+
+#include "common.h"
+
+namespace moe {
+
+namespace {
+
+constexpr int BK = 64;            // k elements per pipeline stage = one 128-byte swizzle span
+constexpr int UMMA_K = 16;        // k elements per tcgen05.mma (bf16)
+constexpr int kBand = 16;         // row tiles that sweep the weight tiles together (L2 reuse)
+constexpr unsigned long long kWaitLimitNs = 4000000000ull;
+constexpr unsigned long long kDrainLimitNs = 2000000ull;
+
+constexpr int kThreads = 192;
+
+// ------------------------------------------------------------------------------ PTX glue
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ unsigned long long gtimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      " .reg .pred p;\n"
+      " mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      " selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = gtimer();
+  unsigned spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 0xffu) == 0) {
+      if (*abort_flag) return false;
+      if (gtimer() - t0 > limit_ns) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                            int c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst),
+               "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulation
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      " .reg .pred p;\n"
+      " setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+        "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+        "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]),
+        "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+        "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+        "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+        "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64
+// elements), written by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_k128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3ffffu) >> 4);  // start address / 16
+  d |= (uint64_t)1 << 16;                    // leading byte offset / 16 (unused with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset / 16
+  d |= (uint64_t)1 << 46;                    // descriptor version of sm_100
+  d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
+__device__ __forceinline__ uint32_t idesc_bf16(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) {
+  return g / (1.0f + __expf(-g)) * u;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+struct Bars {
+  unsigned long long full[8];
+  unsigned long long empty[8];
+  unsigned long long tmem_full[2];
+  unsigned long long tmem_empty[2];
+  unsigned long long drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int NS>
+__device__ __forceinline__ void setup_barriers(Bars& b) {
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(smem_u32(&b.full[s]), 1);
+      mbar_init(smem_u32(&b.empty[s]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&b.tmem_full[i]), 1);
+      mbar_init(smem_u32(&b.tmem_empty[i]), 4);
+    }
+    mbar_init(smem_u32(&b.drain), 1);
+    b.abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+}
+
+// Common tail: after an abort, wait (bounded) for loads and MMAs that are still in flight,
+// report, and release tensor memory.
+template <int NS, int TMEM_COLS>
+__device__ __forceinline__ void teardown(Bars& b, uint32_t tmem_base, uint32_t issued,
+                                         int* status) {
+  tc_fence_before();
+  __syncthreads();
+  const int aborted = *(volatile int*)&b.abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (aborted) {
+    if (warp == 0 && lane == 0) {
+      // the last min(issued, NS) stages may still have a load in flight
+      int dummy = 0;
+      const uint32_t n = issued < (uint32_t)NS ? issued : (uint32_t)NS;
+      for (uint32_t i = 0; i < n; ++i) {
+        const uint32_t it = issued - 1 - i;
+        mbar_wait(smem_u32(&b.full[it % NS]), (it / NS) & 1u, &dummy, kDrainLimitNs);
+      }
+      if (status) atomicExch(status, 1);
+    }
+    if (warp == 1 && lane == 0) {
+      int dummy = 0;
+      umma_commit(smem_u32(&b.drain));
+      mbar_wait(smem_u32(&b.drain), 0, &dummy, kDrainLimitNs);
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------------ gemm_tokens_m
+
+struct TileM {
+  int c, nt, a_row, out_row, rows_valid;
+};
+
+__device__ __forceinline__ void decode_tile_m(const Meta& m, const GemmArgs& a, int item, int Nt,
+                                              TileM& t) {
+  int c = 0;
+  while (c + 1 < a.r && m.tile_prefix[c + 1] * Nt <= item) ++c;
+  const int local = item - m.tile_prefix[c] * Nt;
+  const int Mt = m.tile_prefix[c + 1] - m.tile_prefix[c];
+  const int band = local / (kBand * Nt);
+  const int rem = local - band * kBand * Nt;
+  const int band_rows = min(kBand, Mt - band * kBand);
+  t.nt = rem / band_rows;
+  const int mt = band * kBand + rem - t.nt * band_rows;
+  t.c = c;
+  t.a_row = a.a_row_base + a.a_off_mul * m.off[c] + kTileRows * mt;
+  t.out_row = a.out_row_base + a.out_off_mul * m.off[c] + kTileRows * mt;
+  t.rows_valid = min(kTileRows, m.count[c] - kTileRows * mt);
+}
+
+constexpr int TM_NS = 4;
+constexpr int TM_A_BYTES = 128 * 128;  // 128 token rows x 64 bf16
+constexpr int TM_B_BYTES = 256 * 128;  // 256 weight rows x 64 bf16
+constexpr int TM_STAGE = TM_A_BYTES + TM_B_BYTES;
+constexpr int TM_SMEM = TM_NS * TM_STAGE + 1024;
+constexpr int TM_BN = 256;
+
+template <bool GATE_UP, int OUT>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ Bars bars;
+  __shared__ Meta s_meta;
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
+    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
+  setup_barriers<TM_NS>(bars);
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars.tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *(volatile uint32_t*)&bars.tmem_base;
+  volatile int* abort_flag = &bars.abort_flag;
+
+  const int KB = (args.K + BK - 1) / BK;
+  const int Nt = (args.n_w_rows + TM_BN - 1) / TM_BN;
+  const int n_items = s_meta.tile_prefix[args.r] * Nt;
+  uint32_t issued = 0;
+
+  if (warp == 0) {
+    // ---- TMA producer
+    uint32_t it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      TileM t;
+      decode_tile_m(s_meta, args, item, Nt, t);
+      for (int kb = 0; kb < KB; ++kb, ++it) {
+        const uint32_t s = it % TM_NS, ph = (it / TM_NS) & 1u;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag));
+        if (!ok) break;
+        if (lane == 0) {
+          const uint32_t full = smem_u32(&bars.full[s]);
+          const uint32_t sa = smem_base + s * TM_STAGE;
+          mbar_expect_tx(full, TM_STAGE);
+          tma_load_2d(sa, &maps.t[3], kb * BK, t.a_row, full);
+          tma_load_3d(sa + TM_A_BYTES, &maps.w, kb * BK, t.nt * TM_BN, t.c, full);
+        }
+        __syncwarp();
+      }
+    }
+    issued = it;
+  } else if (warp == 1) {
+    // ---- MMA issuer
+    const uint32_t idesc = idesc_bf16(128, TM_BN);
+    uint32_t it = 0, tile_it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile_it) {
+      const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_empty[buf]), bph ^ 1u, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + buf * TM_BN;
+      for (int kb = 0; kb < KB; ++kb, ++it) {
+        const uint32_t s = it % TM_NS, ph = (it / TM_NS) & 1u;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t sa = smem_base + s * TM_STAGE;
+          const uint64_t adesc = smem_desc_k128(sa);
+          const uint64_t bdesc = smem_desc_k128(sa + TM_A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(smem_u32(&bars.empty[s]));
+          if (kb == KB - 1) umma_commit(smem_u32(&bars.tmem_full[buf]));
+        }
+        __syncwarp();
+      }
+    }
+  } else {
+    // ---- epilogue (warps 2..5): warp w may touch tensor-memory lanes 32*(w%4) .. +31
+    const int wq = warp & 3;
+    const int row = 32 * wq + lane;
+    uint32_t tile_it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile_it) {
+      TileM t;
+      decode_tile_m(s_meta, args, item, Nt, t);
+      const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_full[buf]), bph, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(32 * wq) << 16) + buf * TM_BN;
+      const bool row_ok = row < t.rows_valid;
+      const long long orow = (long long)(t.out_row + row) * args.out_ld + (long long)t.c * args.out_col_mul;
+#pragma unroll 1
+      for (int j = 0; j < TM_BN / 32; ++j) {
+        const int col0 = t.nt * TM_BN + 32 * j;  // first weight row of this chunk
+        if (col0 >= args.n_w_rows) break;        // warp-uniform
+        uint32_t v[32];
+        tmem_ld32(taddr + 32 * j, v);
+        tmem_ld_wait();
+        if (GATE_UP) {
+          // chunk = 16 gate rows then 16 up rows of the features col0/2 .. col0/2 + 15
+          uint32_t o[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float a0 = silu_mul(__uint_as_float(v[2 * i]), __uint_as_float(v[16 + 2 * i]));
+            const float a1 = silu_mul(__uint_as_float(v[2 * i + 1]), __uint_as_float(v[17 + 2 * i]));
+            o[i] = pack_bf16(a0, a1);
+          }
+          if (row_ok) {
+            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(args.out) + orow + (col0 >> 1));
+            dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+            dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+          }
+        } else if (OUT == kOutF32) {
+          if (row_ok) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.out) + orow + col0);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                   __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+          }
+        } else {
+          if (row_ok) {
+            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(args.out) + orow + col0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              dst[i] = make_uint4(
+                  pack_bf16(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
+                  pack_bf16(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
+                  pack_bf16(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
+                  pack_bf16(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[buf]));
+    }
+  }
+  teardown<TM_NS, 512>(bars, tmem_base, issued, args.status);
+}
+
+// ----------------------------------------------------------------------- gemm_weights_m
+
+constexpr int WM_NS = 6;
+constexpr int WM_A_BYTES = 128 * 128;  // 128 weight rows x 64 bf16
+constexpr int WM_B_BYTES = 128 * 128;  // up to 128 token rows x 64 bf16
+constexpr int WM_STAGE = WM_A_BYTES + WM_B_BYTES;
+constexpr int WM_SMEM = WM_NS * WM_STAGE + 1024;
+constexpr int WM_BN = 128;
+
+struct ItemW {
+  int c, mt, ks, tok_row, out_row, cnt, bucket, kb0, kb1;
+};
+
+__device__ __forceinline__ void decode_item_w(const Meta& m, const GemmArgs& a, int item, int Mt,
+                                              int KS, int kb_per_item, int KB, ItemW& w) {
+  const int ks = item % KS;
+  const int rest = item / KS;
+  const int mt = rest % Mt;
+  const int rt = rest / Mt;
+  int c = 0;
+  while (c + 1 < a.r && m.tile_prefix[c + 1] <= rt) ++c;
+  const int n0 = (rt - m.tile_prefix[c]) * WM_BN;
+  w.c = c;
+  w.mt = mt;
+  w.ks = ks;
+  w.cnt = min(WM_BN, m.count[c] - n0);
+  w.bucket = w.cnt <= 16 ? 0 : (w.cnt <= 32 ? 1 : (w.cnt <= 64 ? 2 : 3));
+  w.tok_row = a.a_row_base + a.a_off_mul * m.off[c] + n0;
+  w.out_row = a.out_row_base + a.out_off_mul * m.off[c] + n0;
+  w.kb0 = ks * kb_per_item;
+  w.kb1 = min(KB, w.kb0 + kb_per_item);
+}
+
+template <bool GATE_UP>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args, int kb_per_item) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ Bars bars;
+  __shared__ Meta s_meta;
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
+    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
+  setup_barriers<WM_NS>(bars);
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars.tmem_base), 256);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *(volatile uint32_t*)&bars.tmem_base;
+  volatile int* abort_flag = &bars.abort_flag;
+
+  const int KB = (args.K + BK - 1) / BK;
+  const int KS = (KB + kb_per_item - 1) / kb_per_item;
+  const int Mt = (args.n_w_rows + 127) / 128;
+  const int n_items = s_meta.tile_prefix[args.r] * Mt * KS;
+  uint32_t issued = 0;
+
+  if (warp == 0) {
+    uint32_t it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      ItemW w;
+      decode_item_w(s_meta, args, item, Mt, KS, kb_per_item, KB, w);
+      const uint32_t bytes = WM_A_BYTES + (16u << w.bucket) * 128u;
+      for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+        const uint32_t s = it % WM_NS, ph = (it / WM_NS) & 1u;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag));
+        if (!ok) break;
+        if (lane == 0) {
+          const uint32_t full = smem_u32(&bars.full[s]);
+          const uint32_t sa = smem_base + s * WM_STAGE;
+          mbar_expect_tx(full, bytes);
+          tma_load_3d(sa, &maps.w, kb * BK, w.mt * 128, w.c, full);
+          tma_load_2d(sa + WM_A_BYTES, &maps.t[w.bucket], kb * BK, w.tok_row, full);
+        }
+        __syncwarp();
+      }
+    }
+    issued = it;
+  } else if (warp == 1) {
+    uint32_t it = 0, tile_it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile_it) {
+      ItemW w;
+      decode_item_w(s_meta, args, item, Mt, KS, kb_per_item, KB, w);
+      const uint32_t idesc = idesc_bf16(128, 16 << w.bucket);
+      const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_empty[buf]), bph ^ 1u, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + buf * WM_BN;
+      for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+        const uint32_t s = it % WM_NS, ph = (it / WM_NS) & 1u;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t sa = smem_base + s * WM_STAGE;
+          const uint64_t adesc = smem_desc_k128(sa);
+          const uint64_t bdesc = smem_desc_k128(sa + WM_A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
+          umma_commit(smem_u32(&bars.empty[s]));
+          if (kb == w.kb1 - 1) umma_commit(smem_u32(&bars.tmem_full[buf]));
+        }
+        __syncwarp();
+      }
+    }
+  } else {
+    const int wq = warp & 3;
+    uint32_t tile_it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile_it) {
+      ItemW w;
+      decode_item_w(s_meta, args, item, Mt, KS, kb_per_item, KB, w);
+      const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_full[buf]), bph, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(32 * wq) << 16) + buf * WM_BN;
+      const int wrow = w.mt * 128 + 32 * wq + lane;  // weight row held by this lane
+      const int nchunk = (w.cnt + 15) >> 4;
+      if (GATE_UP) {
+        // lanes 0-15 hold gate rows, lanes 16-31 the up rows of the same 16 features
+        const int feat = (wrow >> 5) * kInterleave + (lane & 15);
+        const bool lane_ok = (lane < 16) && (w.mt * 128 + 32 * wq < args.n_w_rows);
+        bf16* outp = reinterpret_cast<bf16*>(args.out) + (long long)w.out_row * args.out_ld + feat;
+#pragma unroll 1
+        for (int j = 0; j < nchunk; ++j) {
+          uint32_t v[16];
+          tmem_ld16(taddr + 16 * j, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float mine = __uint_as_float(v[i]);
+            const float other = __shfl_xor_sync(0xffffffffu, mine, 16);
+            const int n = 16 * j + i;
+            if (lane_ok && n < w.cnt)
+              outp[(long long)n * args.out_ld] = __float2bfloat16_rn(silu_mul(mine, other));
+          }
+        }
+      } else {
+        const bool lane_ok = wrow < args.n_w_rows;
+        float* outp = reinterpret_cast<float*>(args.out) + (long long)w.ks * args.split_stride +
+                      (long long)w.out_row * args.out_ld + wrow;
+#pragma unroll 1
+        for (int j = 0; j < nchunk; ++j) {
+          uint32_t v[16];
+          tmem_ld16(taddr + 16 * j, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int n = 16 * j + i;
+            if (lane_ok && n < w.cnt) outp[(long long)n * args.out_ld] = __uint_as_float(v[i]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[buf]));
+    }
+  }
+  teardown<WM_NS, 256>(bars, tmem_base, issued, args.status);
+}
+
+// ------------------------------------------------------------ CUDA-core debug kernels
+
+__device__ __forceinline__ float dot8(const uint4& a, const uint4& b, float acc) {
+  const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    acc = fmaf(__uint_as_float(aw[i] << 16), __uint_as_float(bw[i] << 16), acc);
+    acc = fmaf(__uint_as_float(aw[i] & 0xffff0000u), __uint_as_float(bw[i] & 0xffff0000u), acc);
+  }
+  return acc;
+}
+
+__global__ void __launch_bounds__(128)
+simt_gate_up_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W13, GemmArgs a) {
+  const int c = blockIdx.z, i = blockIdx.x;
+  const Meta* m = a.meta;
+  if (i >= m->count[c]) return;
+  const int f = a.n_w_rows / 2, h = a.K;
+  const int j = blockIdx.y * 128 + threadIdx.x;
+  if (j >= f) return;
+  const int q = j / kInterleave, s = j % kInterleave;
+  const long long a_row = a.a_row_base + (long long)a.a_off_mul * m->off[c] + i;
+  const long long o_row = a.out_row_base + (long long)a.out_off_mul * m->off[c] + i;
+  const uint4* xr = reinterpret_cast<const uint4*>(A + a_row * h);
+  const uint4* g = reinterpret_cast<const uint4*>(W13 + ((size_t)c * a.n_w_rows + 32 * q + s) * h);
+  const uint4* u = reinterpret_cast<const uint4*>(W13 + ((size_t)c * a.n_w_rows + 32 * q + 16 + s) * h);
+  float ag = 0.f, au = 0.f;
+  for (int v = 0; v < h / 8; ++v) {
+    const uint4 xv = xr[v];
+    ag = dot8(xv, g[v], ag);
+    au = dot8(xv, u[v], au);
+  }
+  reinterpret_cast<bf16*>(a.out)[o_row * a.out_ld + c * a.out_col_mul + j] =
+      __float2bfloat16_rn(ag / (1.0f + expf(-ag)) * au);
+}
+
+template <int OUT>
+__global__ void __launch_bounds__(128)
+simt_down_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W2, GemmArgs a) {
+  const int c = blockIdx.z, i = blockIdx.x;
+  const Meta* m = a.meta;
+  if (i >= m->count[c]) return;
+  const int h = a.n_w_rows, f = a.K;
+  const int n = blockIdx.y * 128 + threadIdx.x;
+  if (n >= h) return;
+  const long long a_row = a.a_row_base + (long long)a.a_off_mul * m->off[c] + i;
+  const long long o_row = a.out_row_base + (long long)a.out_off_mul * m->off[c] + i;
+  const uint4* ar = reinterpret_cast<const uint4*>(A + a_row * f);
+  const uint4* w = reinterpret_cast<const uint4*>(W2 + ((size_t)c * h + n) * f);
+  float acc = 0.f;
+  for (int v = 0; v < f / 8; ++v) acc = dot8(ar[v], w[v], acc);
+  const long long o = o_row * a.out_ld + c * a.out_col_mul + n;
+  if (OUT == kOutF32) reinterpret_cast<float*>(a.out)[o] = acc;
+  else reinterpret_cast<bf16*>(a.out)[o] = __float2bfloat16_rn(acc);
+}
+
+// ------------------------------------------------------------------------- tensor maps
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+int g_num_sms = 0;
+
+}  // namespace
+
+int gemm_init_driver_api() {
+  if (g_encode) return 0;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess || !fn)
+    return -1;
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return 0;
+}
+
+int make_map_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows) {
+  if (!g_encode) return -1;
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {inner * 2};
+  cuuint32_t box[2] = {BK, box_rows};
+  cuuint32_t es[2] = {1, 1};
+  CUresult rc = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                         strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? 0 : -(int)rc;
+}
+
+int make_map_3d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows, uint64_t planes,
+                uint32_t box_rows) {
+  if (!g_encode) return -1;
+  cuuint64_t dims[3] = {inner, rows, planes};
+  cuuint64_t strides[2] = {inner * 2, inner * rows * 2};
+  cuuint32_t box[3] = {BK, box_rows, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  CUresult rc = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims,
+                         strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? 0 : -(int)rc;
+}
+
+cudaError_t gemm_set_attributes() {
+  cudaError_t e;
+#define SET_ATTR(k, bytes)                                                                 \
+  e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);         \
+  if (e != cudaSuccess) return e;
+  SET_ATTR((gemm_tokens_m_kernel<true, kOutActBf16>), TM_SMEM)
+  SET_ATTR((gemm_tokens_m_kernel<false, kOutF32>), TM_SMEM)
+  SET_ATTR((gemm_tokens_m_kernel<false, kOutBf16>), TM_SMEM)
+  SET_ATTR((gemm_weights_m_kernel<true>), WM_SMEM)
+  SET_ATTR((gemm_weights_m_kernel<false>), WM_SMEM)
+#undef SET_ATTR
+  int dev = 0;
+  e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  return cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+}
+
+cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps& maps,
+                                 const GemmArgs& a, cudaStream_t st) {
+  const int grid = g_num_sms > 0 ? g_num_sms : 148;
+  if (gate_up)
+    gemm_tokens_m_kernel<true, kOutActBf16><<<grid, kThreads, TM_SMEM, st>>>(maps, a);
+  else if (out_kind == kOutF32)
+    gemm_tokens_m_kernel<false, kOutF32><<<grid, kThreads, TM_SMEM, st>>>(maps, a);
+  else
+    gemm_tokens_m_kernel<false, kOutBf16><<<grid, kThreads, TM_SMEM, st>>>(maps, a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
+                                  int kb_per_item, cudaStream_t st) {
+  const int grid = g_num_sms > 0 ? g_num_sms : 148;
+  if (gate_up)
+    gemm_weights_m_kernel<true><<<grid, kThreads, WM_SMEM, st>>>(maps, a, kb_per_item);
+  else
+    gemm_weights_m_kernel<false><<<grid, kThreads, WM_SMEM, st>>>(maps, a, kb_per_item);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,
+                                cudaStream_t st) {
+  const int f = a.n_w_rows / 2;
+  dim3 grid(cap_rows, (f + 127) / 128, a.r);
+  simt_gate_up_kernel<<<grid, 128, 0, st>>>(A, W13, a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_simt_down(const bf16* A, const bf16* W2, const GemmArgs& a, int cap_rows,
+                             GemmOut out_kind, cudaStream_t st) {
+  dim3 grid(cap_rows, (a.n_w_rows + 127) / 128, a.r);
+  if (out_kind == kOutF32) simt_down_kernel<kOutF32><<<grid, 128, 0, st>>>(A, W2, a);
+  else simt_down_kernel<kOutBf16><<<grid, 128, 0, st>>>(A, W2, a);
+  return cudaGetLastError();
+}
+
+}  // namespace moe
