@@ -1,0 +1,596 @@
+// C ABI of libmoe: handle, argument checks, scratch management and the kernel sequences.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <vector>
+
+#include "common.h"
+
+using namespace moe;
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+#define CUDA_TRY(expr)                                                                   \
+  do {                                                                                   \
+    cudaError_t e_ = (expr);                                                             \
+    if (e_ != cudaSuccess)                                                               \
+      return fail(e_ == cudaErrorMemoryAllocation ? MOE_ERR_OOM : MOE_ERR_CUDA, "%s: %s", \
+                  #expr, cudaGetErrorString(e_));                                        \
+  } while (0)
+
+inline int popc(uint32_t v) { return __builtin_popcount(v); }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+long binom(int n, int k) {
+  if (k < 0 || k > n) return 0;
+  long r = 1;
+  for (int i = 1; i <= k; ++i) r = r * (n - k + i) / i;
+  return r;
+}
+
+// A device buffer that only grows.
+struct Buf {
+  void* p = nullptr;
+  size_t bytes = 0;
+};
+
+}  // namespace
+
+// Scratch of the kernel sequences.  Every handle owns one; a stack of layers runs all of
+// its layers out of the first layer's workspace.
+struct Workspace {
+  size_t scratch_bytes = 0;
+  // routing scratch (capacity in tokens)
+  int cap_route_T = 0;
+  Buf idx, wn, ratio, skipped, blk_hist, blk_base, pair_pos, meta, status, sel;
+  // GEMM scratch (capacity in permuted rows)
+  int cap_rows = 0;
+  int map_h = 0, map_f = 0;
+  Buf row_token, xperm, act, O;
+  CUtensorMap tok_x[4], tok_act[4];  // boxes of 16/32/64/128 rows over xperm and act
+  // search scratch
+  Buf s_logits, s_yall, s_act, s_subsets, s_partial, s_loss_sq, s_losses, s_xpad, s_meta;
+  // host staging and stack scratch
+  Buf hx, hy, xn;
+};
+
+struct moe_layer {
+  int h = 0, f = 0, E = 0, r = 0;
+  uint32_t kept_mask = 0;
+  KeptIds kept;
+  bf16* Wg = nullptr;   // [r][h]
+  bf16* W13 = nullptr;  // [r][2f][h], gate/up rows interleaved by 16
+  bf16* W2 = nullptr;   // [r][h][f]
+  size_t weight_bytes = 0;
+  cudaStream_t stream = 0;
+  bool debug_simt = false;
+  CUtensorMap w13_256, w13_128, w2_256, w2_128;
+  Workspace own;
+  Workspace* ws = &own;
+};
+
+namespace {
+
+int grow(moe_layer* L, Buf& b, size_t bytes) {
+  if (bytes <= b.bytes) return MOE_OK;
+  if (b.p) {
+    cudaStreamSynchronize(L->stream);
+    cudaFree(b.p);
+    L->ws->scratch_bytes -= b.bytes;
+    b.p = nullptr;
+    b.bytes = 0;
+  }
+  size_t free_b = 0, total_b = 0;
+  if (cudaMemGetInfo(&free_b, &total_b) == cudaSuccess && bytes > free_b)
+    return fail(MOE_ERR_OOM, "scratch of %zu bytes does not fit (%zu free)", bytes, free_b);
+  cudaError_t e = cudaMalloc(&b.p, bytes);
+  if (e != cudaSuccess) {
+    b.p = nullptr;
+    cudaGetLastError();
+    return fail(MOE_ERR_OOM, "cudaMalloc(%zu): %s", bytes, cudaGetErrorString(e));
+  }
+  b.bytes = bytes;
+  L->ws->scratch_bytes += bytes;
+  return MOE_OK;
+}
+
+void release(moe_layer* L, Buf& b) {
+  if (b.p) cudaFree(b.p);
+  L->own.scratch_bytes -= b.bytes;
+  b.p = nullptr;
+  b.bytes = 0;
+}
+
+int ensure_route(moe_layer* L, int T) {
+  int rc;
+  if ((rc = grow(L, L->ws->meta, sizeof(Meta)))) return rc;
+  if (!L->ws->status.p) {
+    if ((rc = grow(L, L->ws->status, 16))) return rc;
+    CUDA_TRY(cudaMemsetAsync(L->ws->status.p, 0, 16, L->stream));
+  }
+  if ((rc = grow(L, L->ws->sel, 16))) return rc;
+  if (T <= L->ws->cap_route_T) return MOE_OK;
+  const size_t nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
+  if ((rc = grow(L, L->ws->idx, (size_t)T * 8))) return rc;
+  if ((rc = grow(L, L->ws->wn, (size_t)T * 8))) return rc;
+  if ((rc = grow(L, L->ws->ratio, (size_t)T * 4))) return rc;
+  if ((rc = grow(L, L->ws->skipped, align_up((size_t)T, 16)))) return rc;
+  if ((rc = grow(L, L->ws->pair_pos, (size_t)T * 8))) return rc;
+  if ((rc = grow(L, L->ws->blk_hist, nblk * kHistCols * 4))) return rc;
+  if ((rc = grow(L, L->ws->blk_base, nblk * kMaxE * 4))) return rc;
+  L->ws->cap_route_T = T;
+  return MOE_OK;
+}
+
+inline bool decode_mode(int T) { return T <= kDecodeMaxT; }
+inline int rows_for(const moe_layer* L, int T) {
+  const int pad = decode_mode(T) ? 16 : kTileRows;
+  return (int)align_up((size_t)2 * T + (size_t)L->r * pad, 16);
+}
+inline int ksplit_for(const moe_layer* L) {
+  const int KB = (L->f + 63) / 64;
+  return (KB + kDecodeKbPerItem - 1) / kDecodeKbPerItem;
+}
+
+int build_token_maps(GemmMaps& m, const void* base, uint64_t inner, uint64_t rows) {
+  for (int b = 0; b < 4; ++b)
+    if (make_map_2d(&m.t[b], base, inner, rows, 16u << b))
+      return fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed for a token-side operand");
+  return MOE_OK;
+}
+
+int ensure_gemm(moe_layer* L, int T) {
+  // capacity in rows: large enough for this T in its mode, at least 256 (TMA boxes)
+  int need = (int)align_up((size_t)rows_for(L, T), kTileRows) + kTileRows;
+  if (need < 256) need = 256;
+  size_t need_O = (size_t)need * L->h * (decode_mode(T) ? ksplit_for(L) : 1);
+  if (need <= L->ws->cap_rows && need_O * 4 <= L->ws->O.bytes && L->ws->map_h == L->h &&
+      L->ws->map_f == L->f)
+    return MOE_OK;
+  if (need < L->ws->cap_rows) need = L->ws->cap_rows;
+  int rc;
+  if ((rc = grow(L, L->ws->row_token, (size_t)need * 4))) return rc;
+  if ((rc = grow(L, L->ws->xperm, (size_t)need * L->h * 2))) return rc;
+  if ((rc = grow(L, L->ws->act, (size_t)need * L->f * 2))) return rc;
+  if ((rc = grow(L, L->ws->O, need_O * 4))) return rc;
+  L->ws->cap_rows = need;
+  L->ws->map_h = L->h;
+  L->ws->map_f = L->f;
+  GemmMaps tmp;
+  if ((rc = build_token_maps(tmp, L->ws->xperm.p, L->h, need))) return rc;
+  memcpy(L->ws->tok_x, tmp.t, sizeof(tmp.t));
+  if ((rc = build_token_maps(tmp, L->ws->act.p, L->f, need))) return rc;
+  memcpy(L->ws->tok_act, tmp.t, sizeof(tmp.t));
+  return MOE_OK;
+}
+
+int check_status(moe_layer* L) {
+  int st = 0;
+  CUDA_TRY(cudaMemcpyAsync(&st, L->ws->status.p, 4, cudaMemcpyDeviceToHost, L->stream));
+  CUDA_TRY(cudaStreamSynchronize(L->stream));
+  if (st != 0) {
+    cudaMemsetAsync(L->ws->status.p, 0, 4, L->stream);
+    return fail(MOE_ERR_DEVICE_TIMEOUT, "a bounded wait inside a GEMM kernel expired");
+  }
+  return MOE_OK;
+}
+
+// The two grouped GEMMs of the experts over a batch described by `meta`.
+int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmMaps& m_gu,
+                     const GemmMaps& m_dn, GemmArgs gu, GemmArgs dn, GemmOut dn_kind,
+                     const bf16* gu_A, const bf16* dn_A, int simt_rows) {
+  gu.meta = meta; dn.meta = meta;
+  gu.r = L->r; dn.r = L->r;
+  gu.K = L->h; gu.n_w_rows = 2 * L->f;
+  dn.K = L->f; dn.n_w_rows = L->h;
+  gu.status = (int*)L->ws->status.p; dn.status = (int*)L->ws->status.p;
+  if (L->debug_simt) {
+    CUDA_TRY(launch_simt_gate_up(gu_A, L->W13, gu, simt_rows, L->stream));
+    CUDA_TRY(launch_simt_down(dn_A, L->W2, dn, simt_rows, dn_kind, L->stream));
+  } else if (weights_m) {
+    CUDA_TRY(launch_gemm_weights_m(true, m_gu, gu, (L->h + 63) / 64, L->stream));
+    CUDA_TRY(launch_gemm_weights_m(false, m_dn, dn, kDecodeKbPerItem, L->stream));
+  } else {
+    CUDA_TRY(launch_gemm_tokens_m(true, kOutActBf16, m_gu, gu, L->stream));
+    CUDA_TRY(launch_gemm_tokens_m(false, dn_kind, m_dn, dn, L->stream));
+  }
+  return MOE_OK;
+}
+
+int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* residual, void* y,
+                 void* stats) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
+  if (T == 0) return MOE_OK;
+  if (!x || !y) return fail(MOE_ERR_INVALID_ARG, "x or y is NULL");
+  if (!aligned16(x) || !aligned16(y) || !aligned16(residual) || !aligned16(stats))
+    return fail(MOE_ERR_INVALID_ARG, "x, y, residual and routing_stats must be 16-byte aligned");
+  if (!(beta >= 0.f)) return fail(MOE_ERR_INVALID_ARG, "beta must be >= 0");
+  if (x == y) return fail(MOE_ERR_INVALID_ARG, "x and y may not overlap");
+  int rc;
+  if ((rc = ensure_route(L, T))) return rc;
+  if ((rc = ensure_gemm(L, T))) return rc;
+  cudaStream_t st = L->stream;
+  const bool dec = decode_mode(T);
+  const int nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
+  const int rows_cap = rows_for(L, T);
+
+  RouteOut ro;
+  memset(&ro, 0, sizeof(ro));
+  ro.idx = (int32_t*)L->ws->idx.p; ro.wn = (float*)L->ws->wn.p; ro.ratio = (float*)L->ws->ratio.p;
+  ro.skipped = (uint8_t*)L->ws->skipped.p; ro.blk_hist = (int32_t*)L->ws->blk_hist.p;
+  int32_t *s_count = nullptr, *s_nsk = nullptr, *s_nt = nullptr;
+  if (stats) {
+    size_t off[7];
+    moe_routing_stats_layout(T, L->E, off);
+    char* s = (char*)stats;
+    ro.s_idx = (int32_t*)(s + off[0]); ro.s_wn = (float*)(s + off[1]);
+    ro.s_ratio = (float*)(s + off[2]); ro.s_skipped = (uint8_t*)(s + off[3]);
+    s_count = (int32_t*)(s + off[4]); s_nsk = (int32_t*)(s + off[5]); s_nt = (int32_t*)(s + off[6]);
+  }
+  Meta* meta = (Meta*)L->ws->meta.p;
+  CUDA_TRY(launch_router((const bf16*)x, L->Wg, T, L->h, L->r, beta, L->kept, ro, st));
+  CUDA_TRY(launch_scan(ro.blk_hist, nblk, L->r, dec ? 16 : kTileRows, (int32_t*)L->ws->blk_base.p, meta,
+                       s_count, s_nsk, s_nt, L->kept, L->E, st));
+  CUDA_TRY(cudaMemsetAsync(L->ws->row_token.p, 0xff, (size_t)rows_cap * 4, st));
+  CUDA_TRY(launch_scatter(ro.idx, ro.skipped, (int32_t*)L->ws->blk_base.p, meta, T,
+                          (int32_t*)L->ws->pair_pos.p, (int32_t*)L->ws->row_token.p, st));
+  CUDA_TRY(launch_gather((const bf16*)x, (int32_t*)L->ws->row_token.p, meta, L->h, rows_cap,
+                         (bf16*)L->ws->xperm.p, st));
+
+  GemmArgs gu, dn;
+  memset(&gu, 0, sizeof(gu));
+  memset(&dn, 0, sizeof(dn));
+  gu.a_off_mul = 1; gu.out_off_mul = 1; gu.out_ld = L->f; gu.out = L->ws->act.p;
+  dn.a_off_mul = 1; dn.out_off_mul = 1; dn.out_ld = L->h; dn.out = L->ws->O.p;
+  const bool wm = dec && !L->debug_simt;
+  const int ksplit = wm ? ksplit_for(L) : 1;
+  const size_t split_stride = (size_t)rows_cap * L->h;
+  dn.split_stride = (long long)split_stride;
+  GemmMaps m_gu, m_dn;
+  m_gu.w = wm ? L->w13_128 : L->w13_256;
+  m_dn.w = wm ? L->w2_128 : L->w2_256;
+  memcpy(m_gu.t, L->ws->tok_x, sizeof(m_gu.t));
+  memcpy(m_dn.t, L->ws->tok_act, sizeof(m_dn.t));
+  rc = run_expert_gemms(L, meta, wm, m_gu, m_dn, gu, dn, kOutF32, (const bf16*)L->ws->xperm.p,
+                        (const bf16*)L->ws->act.p, rows_cap);
+  if (rc) return rc;
+  CUDA_TRY(launch_combine((const float*)L->ws->O.p, ksplit, split_stride, (int32_t*)L->ws->pair_pos.p,
+                          (float*)L->ws->wn.p, (const bf16*)residual, T, L->h, (bf16*)y, st));
+  return MOE_OK;
+}
+
+}  // namespace
+
+// ======================================================================================
+extern "C" {
+
+const char* moe_last_error(void) { return g_err; }
+
+long moe_num_subsets(int E, int r) {
+  if (E < 2 || E > kMaxE || r < 2 || r > E) return 0;
+  return binom(E, r);
+}
+
+size_t moe_routing_stats_layout(int T, int E, size_t offsets[7]) {
+  size_t o = 0;
+  const size_t sizes[7] = {(size_t)T * 8, (size_t)T * 8, (size_t)T * 4, (size_t)T,
+                           (size_t)E * 8, 4, 4};
+  for (int i = 0; i < 7; ++i) {
+    if (offsets) offsets[i] = o;
+    o = align_up(o + sizes[i], 16);
+  }
+  return o;
+}
+
+size_t moe_routing_stats_bytes(int T, int E) { return moe_routing_stats_layout(T, E, nullptr); }
+
+moe_layer_t* moe_layer_create(const void* W_gate, const void* W1, const void* W3, const void* W2,
+                              int h, int f, int E, uint32_t kept_mask) {
+  g_err[0] = 0;
+  if (!W_gate || !W1 || !W3 || !W2) { fail(MOE_ERR_INVALID_ARG, "a weight pointer is NULL"); return nullptr; }
+  if (!aligned16(W_gate) || !aligned16(W1) || !aligned16(W3) || !aligned16(W2)) {
+    fail(MOE_ERR_INVALID_ARG, "weight pointers must be 16-byte aligned");
+    return nullptr;
+  }
+  if (E < 2 || E > kMaxE) { fail(MOE_ERR_UNSUPPORTED_SHAPE, "E = %d outside 2..%d", E, kMaxE); return nullptr; }
+  if (h < 64 || f < 64 || h % 64 || f % 64) {
+    fail(MOE_ERR_UNSUPPORTED_SHAPE, "h = %d and f = %d must be positive multiples of 64", h, f);
+    return nullptr;
+  }
+  if (kept_mask >> E) { fail(MOE_ERR_INVALID_ARG, "kept_mask has bits beyond expert %d", E - 1); return nullptr; }
+  if (popc(kept_mask) < 2) { fail(MOE_ERR_INVALID_ARG, "kept_mask keeps fewer than 2 experts"); return nullptr; }
+
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+    cudaGetLastError();
+    fail(MOE_ERR_CUDA, "no usable CUDA device");
+    return nullptr;
+  }
+  if (major != 10) { fail(MOE_ERR_ARCH, "device has compute capability %d.x, sm_100 is required", major); return nullptr; }
+  if (gemm_init_driver_api()) { fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled is not available"); return nullptr; }
+  cudaError_t e = gemm_set_attributes();
+  if (e != cudaSuccess) { fail(MOE_ERR_CUDA, "kernel attributes: %s", cudaGetErrorString(e)); return nullptr; }
+
+  moe_layer* L = new (std::nothrow) moe_layer();
+  if (!L) { fail(MOE_ERR_OOM, "host allocation failed"); return nullptr; }
+  L->h = h; L->f = f; L->E = E; L->kept_mask = kept_mask; L->r = popc(kept_mask);
+  for (int e_ = 0, c = 0; e_ < kMaxE; ++e_) {
+    if (e_ < E && ((kept_mask >> e_) & 1u)) L->kept.id[c++] = e_;
+  }
+  for (int c = L->r; c < kMaxE; ++c) L->kept.id[c] = 0;
+  const char* dbg = getenv("MOE_DEBUG_SIMT");
+  L->debug_simt = dbg && dbg[0] == '1';
+
+  const size_t n_gate = (size_t)L->r * h * 2, n_13 = (size_t)L->r * 2 * f * h * 2,
+               n_2 = (size_t)L->r * h * f * 2;
+  size_t free_b = 0, total_b = 0;
+  cudaMemGetInfo(&free_b, &total_b);
+  if (n_gate + n_13 + n_2 > free_b) {
+    fail(MOE_ERR_OOM, "weights of %zu bytes do not fit (%zu free)", n_gate + n_13 + n_2, free_b);
+    delete L;
+    return nullptr;
+  }
+  bool ok = cudaMalloc((void**)&L->Wg, n_gate) == cudaSuccess &&
+            cudaMalloc((void**)&L->W13, n_13) == cudaSuccess &&
+            cudaMalloc((void**)&L->W2, n_2) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    fail(MOE_ERR_OOM, "cudaMalloc of the layer weights failed");
+    moe_layer_destroy(L);
+    return nullptr;
+  }
+  L->weight_bytes = n_gate + n_13 + n_2;
+  for (int c = 0; c < L->r && ok; ++c) {
+    const int id = L->kept.id[c];
+    ok = ok && cudaMemcpyAsync(L->Wg + (size_t)c * h, (const bf16*)W_gate + (size_t)id * h,
+                               (size_t)h * 2, cudaMemcpyDeviceToDevice, 0) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(L->W2 + (size_t)c * h * f, (const bf16*)W2 + (size_t)id * h * f,
+                               (size_t)h * f * 2, cudaMemcpyDeviceToDevice, 0) == cudaSuccess;
+  }
+  ok = ok && launch_interleave((const bf16*)W1, (const bf16*)W3, L->kept, L->r, f, h, L->W13, 0) ==
+                 cudaSuccess;
+  ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+  if (!ok) {
+    fail(MOE_ERR_CUDA, "copying the weights failed: %s", cudaGetErrorString(cudaGetLastError()));
+    moe_layer_destroy(L);
+    return nullptr;
+  }
+  if (make_map_3d(&L->w13_256, L->W13, h, 2 * (uint64_t)f, L->r, 256) ||
+      make_map_3d(&L->w13_128, L->W13, h, 2 * (uint64_t)f, L->r, 128) ||
+      make_map_3d(&L->w2_256, L->W2, f, h, L->r, 256) ||
+      make_map_3d(&L->w2_128, L->W2, f, h, L->r, 128)) {
+    fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled failed for the weights");
+    moe_layer_destroy(L);
+    return nullptr;
+  }
+  return L;
+}
+
+void moe_layer_destroy(moe_layer_t* L) {
+  if (!L) return;
+  cudaStreamSynchronize(L->stream);
+  Buf* bufs[] = {&L->own.idx, &L->own.wn, &L->own.ratio, &L->own.skipped, &L->own.blk_hist, &L->own.blk_base, &L->own.pair_pos,
+                 &L->own.meta, &L->own.status, &L->own.sel, &L->own.row_token, &L->own.xperm, &L->own.act, &L->own.O,
+                 &L->own.s_logits, &L->own.s_yall, &L->own.s_act, &L->own.s_subsets, &L->own.s_partial, &L->own.s_loss_sq,
+                 &L->own.s_losses, &L->own.s_xpad, &L->own.s_meta, &L->own.hx, &L->own.hy, &L->own.xn};
+  for (Buf* b : bufs) release(L, *b);
+  if (L->Wg) cudaFree(L->Wg);
+  if (L->W13) cudaFree(L->W13);
+  if (L->W2) cudaFree(L->W2);
+  delete L;
+}
+
+int moe_set_stream(moe_layer_t* L, void* cuda_stream) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  L->stream = (cudaStream_t)cuda_stream;
+  return MOE_OK;
+}
+
+size_t moe_layer_weight_bytes(const moe_layer_t* L) { return L ? L->weight_bytes : 0; }
+size_t moe_layer_scratch_bytes(const moe_layer_t* L) { return L ? L->own.scratch_bytes : 0; }
+
+int moe_forward(moe_layer_t* L, const void* x, int T, float beta, void* y, void* routing_stats) {
+  return forward_impl(L, x, T, beta, nullptr, y, routing_stats);
+}
+
+int moe_forward_residual(moe_layer_t* L, const void* x, int T, float beta, const void* residual,
+                         void* y, void* routing_stats) {
+  return forward_impl(L, x, T, beta, residual, y, routing_stats);
+}
+
+int moe_forward_host(moe_layer_t* L, const void* x_host, int T, float beta, void* y_host) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
+  if (T == 0) return MOE_OK;
+  if (!x_host || !y_host) return fail(MOE_ERR_INVALID_ARG, "x_host or y_host is NULL");
+  const size_t bytes = (size_t)T * L->h * 2;
+  int rc;
+  if ((rc = grow(L, L->ws->hx, bytes))) return rc;
+  if ((rc = grow(L, L->ws->hy, bytes))) return rc;
+  CUDA_TRY(cudaMemcpyAsync(L->ws->hx.p, x_host, bytes, cudaMemcpyHostToDevice, L->stream));
+  if ((rc = forward_impl(L, L->ws->hx.p, T, beta, nullptr, L->ws->hy.p, nullptr))) return rc;
+  CUDA_TRY(cudaMemcpyAsync(y_host, L->ws->hy.p, bytes, cudaMemcpyDeviceToHost, L->stream));
+  return check_status(L);
+}
+
+int moe_calibrate_beta(moe_layer_t* L, const void* x, int T, float* beta_out) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  if (!x || !beta_out) return fail(MOE_ERR_INVALID_ARG, "x or beta_out is NULL");
+  if (T < 1) return fail(MOE_ERR_INVALID_ARG, "T = %d: at least one calibration token is needed", T);
+  if (!aligned16(x)) return fail(MOE_ERR_INVALID_ARG, "x must be 16-byte aligned");
+  int rc;
+  if ((rc = ensure_route(L, T))) return rc;
+  RouteOut ro;
+  memset(&ro, 0, sizeof(ro));
+  ro.idx = (int32_t*)L->ws->idx.p; ro.wn = (float*)L->ws->wn.p; ro.ratio = (float*)L->ws->ratio.p;
+  ro.skipped = (uint8_t*)L->ws->skipped.p;
+  CUDA_TRY(launch_router((const bf16*)x, L->Wg, T, L->h, L->r, 0.f, L->kept, ro, L->stream));
+  CUDA_TRY(launch_select2(ro.ratio, T, (T - 1) / 2, T / 2, (float*)L->ws->sel.p, L->stream));
+  float v[2];
+  CUDA_TRY(cudaMemcpyAsync(v, L->ws->sel.p, 8, cudaMemcpyDeviceToHost, L->stream));
+  CUDA_TRY(cudaStreamSynchronize(L->stream));
+  *beta_out = (T & 1) ? v[0] : (float)(((double)v[0] + (double)v[1]) * 0.5);
+  return MOE_OK;
+}
+
+int moe_prune_search(moe_layer_t* L, const void* x_calib, int T, int r, float* losses,
+                     uint32_t* best_subset) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  if (!x_calib || !losses || !best_subset)
+    return fail(MOE_ERR_INVALID_ARG, "x_calib, losses or best_subset is NULL");
+  if (!aligned16(x_calib)) return fail(MOE_ERR_INVALID_ARG, "x_calib must be 16-byte aligned");
+  if (T < 1) return fail(MOE_ERR_INVALID_ARG, "T = %d: at least one calibration token is needed", T);
+  if (L->r != L->E)
+    return fail(MOE_ERR_INVALID_ARG, "the search needs a layer created with all %d experts kept", L->E);
+  if (r < 2 || r > L->E) return fail(MOE_ERR_INVALID_ARG, "r = %d outside 2..%d", r, L->E);
+  const int E = L->E, h = L->h, f = L->f;
+  const long nC = binom(E, r);
+  cudaStream_t st = L->stream;
+  int rc;
+  if ((rc = ensure_route(L, T))) return rc;
+
+  // subsets in lexicographic order of their ascending index tuples
+  std::vector<uint32_t> masks;
+  masks.reserve(nC);
+  {
+    int c[kMaxE];
+    for (int i = 0; i < r; ++i) c[i] = i;
+    for (;;) {
+      uint32_t m = 0;
+      for (int i = 0; i < r; ++i) m |= 1u << c[i];
+      masks.push_back(m);
+      int i = r - 1;
+      while (i >= 0 && c[i] == E - r + i) --i;
+      if (i < 0) break;
+      ++c[i];
+      for (int j = i + 1; j < r; ++j) c[j] = c[j - 1] + 1;
+    }
+  }
+
+  const int Tc = T < 8192 ? T : 8192;                     // tokens per all-experts chunk
+  const int Tc_pad = (int)align_up((size_t)Tc, kTileRows);
+  const int nblk_enum = enumerate_num_blocks(T, (int)nC);
+  if ((rc = grow(L, L->ws->s_logits, (size_t)T * E * 4))) return rc;
+  if ((rc = grow(L, L->ws->s_yall, (size_t)T * E * h * 2))) return rc;
+  if ((rc = grow(L, L->ws->s_act, ((size_t)E * Tc_pad + kTileRows) * f * 2))) return rc;
+  if ((rc = grow(L, L->ws->s_subsets, (size_t)nC * 4))) return rc;
+  if ((rc = grow(L, L->ws->s_partial, (size_t)nblk_enum * nC * 4))) return rc;
+  if ((rc = grow(L, L->ws->s_loss_sq, (size_t)nC * 8))) return rc;
+  if ((rc = grow(L, L->ws->s_losses, (size_t)nC * 4))) return rc;
+  if ((rc = grow(L, L->ws->s_meta, sizeof(Meta)))) return rc;
+  CUDA_TRY(cudaMemcpyAsync(L->ws->s_subsets.p, masks.data(), (size_t)nC * 4, cudaMemcpyHostToDevice, st));
+
+  // token-side operand of the gate/up GEMM: x itself (padded copy when shorter than one box)
+  const bf16* xa = (const bf16*)x_calib;
+  uint64_t xa_rows = (uint64_t)T;
+  if (T < kTileRows) {
+    if ((rc = grow(L, L->ws->s_xpad, (size_t)kTileRows * h * 2))) return rc;
+    CUDA_TRY(cudaMemsetAsync(L->ws->s_xpad.p, 0, (size_t)kTileRows * h * 2, st));
+    CUDA_TRY(cudaMemcpyAsync(L->ws->s_xpad.p, x_calib, (size_t)T * h * 2, cudaMemcpyDeviceToDevice, st));
+    xa = (const bf16*)L->ws->s_xpad.p;
+    xa_rows = kTileRows;
+  }
+  GemmMaps m_gu, m_dn;
+  m_gu.w = L->w13_256;
+  m_dn.w = L->w2_256;
+  if ((rc = build_token_maps(m_gu, xa, h, xa_rows))) return rc;
+  if ((rc = build_token_maps(m_dn, L->ws->s_act.p, f, (uint64_t)E * Tc_pad + kTileRows))) return rc;
+
+  // all logits (Sec. 3.2: the unpruned layer's routing), then every expert on every token
+  RouteOut ro;
+  memset(&ro, 0, sizeof(ro));
+  ro.idx = (int32_t*)L->ws->idx.p; ro.wn = (float*)L->ws->wn.p; ro.ratio = (float*)L->ws->ratio.p;
+  ro.skipped = (uint8_t*)L->ws->skipped.p; ro.logits = (float*)L->ws->s_logits.p;
+  CUDA_TRY(launch_router((const bf16*)x_calib, L->Wg, T, h, E, 0.f, L->kept, ro, st));
+  Meta* meta = (Meta*)L->ws->s_meta.p;
+  for (int t0 = 0; t0 < T; t0 += Tc) {
+    const int rows = (T - t0) < Tc ? (T - t0) : Tc;
+    CUDA_TRY(launch_set_dense_meta(meta, E, rows, Tc_pad, st));
+    GemmArgs gu, dn;
+    memset(&gu, 0, sizeof(gu));
+    memset(&dn, 0, sizeof(dn));
+    gu.a_row_base = t0; gu.a_off_mul = 0; gu.out_off_mul = 1; gu.out_ld = f; gu.out = L->ws->s_act.p;
+    dn.a_off_mul = 1; dn.out_row_base = t0; dn.out_off_mul = 0; dn.out_col_mul = h;
+    dn.out_ld = (long long)E * h; dn.out = L->ws->s_yall.p;
+    if ((rc = run_expert_gemms(L, meta, false, m_gu, m_dn, gu, dn, kOutBf16, xa,
+                               (const bf16*)L->ws->s_act.p, rows)))
+      return rc;
+  }
+  CUDA_TRY(launch_enumerate((const float*)L->ws->s_logits.p, (const bf16*)L->ws->s_yall.p, T, E, r, h,
+                            (const uint32_t*)L->ws->s_subsets.p, (int)nC, (float*)L->ws->s_partial.p,
+                            (double*)L->ws->s_loss_sq.p, (float*)L->ws->s_losses.p, st));
+  CUDA_TRY(cudaMemcpyAsync(losses, L->ws->s_losses.p, (size_t)nC * 4, cudaMemcpyDeviceToHost, st));
+  if ((rc = check_status(L))) return rc;
+  long best = 0;
+  for (long c = 1; c < nC; ++c)
+    if (losses[c] < losses[best]) best = c;
+  *best_subset = masks[best];
+  return MOE_OK;
+}
+
+int moe_rmsnorm(const void* x, int T, int h, float eps, void* out, void* cuda_stream) {
+  if (T < 0 || h < 8 || h % 8) return fail(MOE_ERR_INVALID_ARG, "bad T = %d or h = %d", T, h);
+  if (T == 0) return MOE_OK;
+  if (!x || !out || !aligned16(x) || !aligned16(out))
+    return fail(MOE_ERR_INVALID_ARG, "x and out must be non-NULL and 16-byte aligned");
+  CUDA_TRY(launch_rmsnorm((const bf16*)x, T, h, eps, (bf16*)out, (cudaStream_t)cuda_stream));
+  return MOE_OK;
+}
+
+int moe_stack_forward(moe_layer_t* const* layers, int n_layers, const void* x, int T,
+                      const float* betas, float eps, void* y) {
+  if (!layers || n_layers < 1) return fail(MOE_ERR_INVALID_ARG, "no layers");
+  if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
+  if (T == 0) return MOE_OK;
+  if (!x || !y || x == y) return fail(MOE_ERR_INVALID_ARG, "x and y must be distinct and non-NULL");
+  moe_layer* L0 = layers[0];
+  if (!L0) return fail(MOE_ERR_INVALID_ARG, "layer 0 is NULL");
+  for (int l = 0; l < n_layers; ++l)
+    if (!layers[l] || layers[l]->h != L0->h)
+      return fail(MOE_ERR_INVALID_ARG, "layer %d is NULL or has a different h", l);
+  int rc;
+  if ((rc = grow(L0, L0->ws->xn, (size_t)T * L0->h * 2))) return rc;
+  const void* cur = x;
+  for (int l = 0; l < n_layers; ++l) {
+    moe_layer* L = layers[l];
+    cudaStream_t saved = L->stream;
+    L->stream = L0->stream;
+    L->ws = (L->f == L0->f) ? &L0->own : &L->own;
+    rc = MOE_OK;
+    cudaError_t e = launch_rmsnorm((const bf16*)cur, T, L->h, eps, (bf16*)L0->ws->xn.p, L0->stream);
+    if (e != cudaSuccess) rc = fail(MOE_ERR_CUDA, "rmsnorm: %s", cudaGetErrorString(e));
+    if (!rc) rc = forward_impl(L, L0->ws->xn.p, T, betas ? betas[l] : 0.f, cur, y, nullptr);
+    L->stream = saved;
+    L->ws = &L->own;
+    if (rc) return rc;
+    cur = y;
+  }
+  return MOE_OK;
+}
+
+int moe_device_status(moe_layer_t* L) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  if (!L->ws->status.p) {
+    CUDA_TRY(cudaStreamSynchronize(L->stream));
+    return MOE_OK;
+  }
+  return check_status(L);
+}
+
+}  // extern "C"

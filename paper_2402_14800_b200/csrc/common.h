@@ -118,7 +118,7 @@ cudaError_t launch_simt_down(const bf16* A, const bf16* W2, const GemmArgs& a, i
 cudaError_t gemm_set_attributes();
 
 // ---- search (search.cu) ---------------------------------------------------------------
-int enumerate_num_blocks(int T);
+int enumerate_num_blocks(int T, int nC);
 cudaError_t launch_enumerate(const float* logits, const bf16* Yall, int T, int E, int r, int h,
                              const uint32_t* subsets, int nC, float* partial, double* loss_sq,
                              float* losses, cudaStream_t st);
