@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE layer hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload decode|prefill|search]
+                    [--tokens T] [--beta calibrated|0] [--kept full|r6|r4] [--impl ours|reference]
+
+One step = one pass of the whole hot path (router, permutation, both grouped GEMMs, combine;
+or the pruning search) over one batch of seeded synthetic tokens at the Mixtral-8x7B layer
+shape.  Prints ONE JSON line.  With N > 1 (launched by torch.distributed.run) every rank runs
+an independent replica on its own GPU: the path has no exchange step, so no collective sits
+on the data path; timing is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2402_14800_b200 import synth  # noqa: E402
+
+H, F, E = synth.MIXTRAL["h"], synth.MIXTRAL["f"], synth.MIXTRAL["E"]
+FLOP_PER_PAIR = 2 * 3 * H * F
+KEPT = {"full": 0xFF, "r6": 0x3F, "r4": 0x0F}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=float(d["hbm_gbs"]), tf_burst=float(d["bf16_tflops"]),
+                    tf_sust=float(d["bf16_tflops_sustained"]), source="measured")
+    return dict(hbm=6650.0, tf_burst=1590.0, tf_sust=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def workload_name(a):
+    if a.workload == "search":
+        return "search_T%d_r%s" % (a.tokens, a.search_r)
+    return "%s_T%d_%s_beta-%s" % (a.workload, a.tokens, a.kept, a.beta)
+
+
+# ------------------------------------------------------------------------- reference arm
+
+def oracle_sample(a, W_host, x_host, beta, n_sample):
+    from oracle import moe_oracle as O
+    xs = x_host[:n_sample]
+    t0 = time.perf_counter()
+    if a.workload == "search":
+        for r in (6, 4):
+            O.prune_search_allexperts(xs, W_host["Wg"], W_host["W1"], W_host["W3"], W_host["W2"], r)
+    else:
+        O.moe_forward(xs, W_host["Wg"], W_host["W1"], W_host["W3"], W_host["W2"], KEPT[a.kept], beta)
+    return time.perf_counter() - t0
+
+
+def units_per_step(a):
+    # tokens for the forward workloads; subsets x tokens for the search (28 + 70 subsets)
+    return a.tokens * (98 if a.workload == "search" else 1)
+
+
+def metric_unit(a):
+    if a.workload == "search":
+        return "pruning-search subsets*tokens/s on 1 B200 (Mixtral-shaped layer, r=6 and r=4)", "subsets*tokens/s"
+    return "MoE-layer tokens/s on 1 B200 (decode/prefill, +-skip/prune); % HBM or bf16 peak", "tokens/s"
+
+
+def host_inputs(a, device):
+    """Weights, tokens and the calibration batch; drawn on `device`, copies on the host."""
+    W = synth.make_layer_weights(H, F, E, seed=0, device=device)
+    x = synth.make_tokens(a.tokens, H, seed=1, device=device)
+    xcal = synth.make_tokens(4096, H, seed=1001, device=device)
+    return W, x, xcal
+
+
+def run_reference(a):
+    rank, world, local = dist_env()
+    if rank != 0:
+        return 0
+    from oracle import moe_oracle as O
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    W, x, xcal = host_inputs(a, dev)
+    b = synth.bf16_bits
+    Wh = dict(Wg=b(W.W_gate), W1=b(W.W1), W3=b(W.W3), W2=b(W.W2))
+    xh = b(x)
+    beta = 0.0
+    if a.beta == "calibrated" and a.workload != "search":
+        beta = O.beta_median(O.route(b(xcal), Wh["Wg"], KEPT[a.kept], 0.0)["ratio"])
+    del W
+    # size the per-step sample from a probe so that K steps take about a minute in total
+    probe = 2
+    dt = oracle_sample(a, Wh, xh, beta, probe)
+    budget_s = 60.0
+    n_sample = int(max(1, min(a.tokens, 128, budget_s / max(a.steps, 1) / (dt / probe))))
+    for _ in range(min(a.warmup, 1)):
+        oracle_sample(a, Wh, xh, beta, 1)
+    times = [oracle_sample(a, Wh, xh, beta, n_sample) for _ in range(a.steps)]
+    per_unit = (98 if a.workload == "search" else 1)
+    value = n_sample * per_unit * a.steps / sum(times)
+    metric, unit = metric_unit(a)
+    sample = "%d of %d tokens per step, oracle as it stands" % (n_sample, a.tokens)
+    line = {
+        "impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": a.gpus,
+        "steps": a.steps, "warmup": a.warmup, "ms_per_step": 1e3 * sum(times) / a.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": workload_name(a), "h": H, "f": F, "E": E, "beta": beta},
+        "cpu_baseline": {"value": value, "unit": unit, "cores": O.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# -------------------------------------------------------------------------------- our arm
+
+def run_ours(a):
+    from paper_2402_14800_b200 import binding, build
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (sm_100a); there is no CPU fallback")
+    build.build()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = measured_peaks()
+
+    W, x, xcal = host_inputs(a, dev)
+    kept = KEPT[a.kept]
+    layer = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, kept if a.workload != "search" else 0xFF)
+    stream = torch.cuda.Stream(dev)
+    layer.set_stream(stream)
+    beta = 0.0
+    if a.beta == "calibrated" and a.workload != "search":
+        beta = layer.calibrate_beta(xcal)
+    T = a.tokens
+    y = torch.empty_like(x)
+    stats = binding.RoutingStats(T, E, dev)
+
+    if a.workload == "search":
+        def step():
+            layer.prune_search(x, 6)
+            layer.prune_search(x, 4)
+        launches_per_step = None
+    else:
+        def step():
+            layer.forward(x, beta, y=y)
+        launches_per_step = 7  # router, scan, scatter, gather, gate/up GEMM, down GEMM, combine
+
+    # routing facts for the algorithmic byte / flop counts (one untimed call)
+    pairs = touched = 0
+    if a.workload != "search":
+        layer.forward(x, beta, y=y, stats=stats)
+        stream.synchronize()
+        pairs = 2 * T - int(stats.n_skipped.item())
+        touched = int(stats.n_experts_touched.item())
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(a.warmup, 3)):
+            step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    if a.workload != "search":
+        layer.profile_enable(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with torch.cuda.stream(stream):
+        ev0.record(stream)
+        for _ in range(a.steps):
+            step()
+        ev1.record(stream)
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    stage_ms, ncalls = ([0, 0, 0, 0], 0)
+    if a.workload != "search":
+        stage_ms, ncalls = layer.profile_read()
+        layer.profile_enable(False)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / a.steps
+    value = world * units_per_step(a) * a.steps / (ms_total * 1e-3)
+
+    # end to end through the host-buffer entry point (forward workloads only)
+    e2e = None
+    if a.workload != "search":
+        xh = x.cpu().pin_memory()
+        yh = torch.empty_like(xh).pin_memory()
+        for _ in range(3):
+            layer.forward_host(xh, beta, yh)
+        barrier()
+        t0 = time.perf_counter()
+        n_e2e = max(3, min(a.steps, 50))
+        for _ in range(n_e2e):
+            layer.forward_host(xh, beta, yh)
+        torch.cuda.synchronize(dev)
+        dt = time.perf_counter() - t0
+        if world > 1:
+            import torch.distributed as dist
+            tt = torch.tensor([dt], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            dt = float(tt.item())
+        e2e = {"value": world * T * n_e2e / dt, "unit": "tokens/s", "h2d_bytes_per_step": T * H * 2,
+               "d2h_bytes_per_step": T * H * 2, "timing": "host wall clock around the C-ABI call, max over ranks"}
+    else:
+        # the search already returns its losses to host memory inside the timed call
+        e2e = {"value": value, "unit": "subsets*tokens/s", "h2d_bytes_per_step": 0,
+               "d2h_bytes_per_step": 98 * 4 + 8,
+               "timing": "inputs resident on device; losses and argmin are copied to the host inside the call"}
+
+    # roofline of the dominant kernel (gate/up grouped GEMM), from the live per-stage events
+    roofline = None
+    stages = None
+    if a.workload != "search" and ncalls > 0:
+        gu_ms = stage_ms[1] / ncalls
+        dn_ms = stage_ms[2] / ncalls
+        stages = {"route_permute_ms": stage_ms[0] / ncalls, "gate_up_ms": gu_ms, "down_ms": dn_ms,
+                  "combine_ms": stage_ms[3] / ncalls}
+        if a.workload == "decode":
+            gu_bytes = touched * 2 * F * H * 2 + pairs * H * 2 + pairs * F * 2
+            dn_bytes = touched * H * F * 2 + pairs * F * 2 + 7 * pairs * H * 4
+            ach = gu_bytes / (gu_ms * 1e-3) / 1e9
+            roofline = {"bound": "hbm", "kernel": "gemm_weights_m_kernel<gate_up>", "achieved": ach,
+                        "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"], "traffic": None,
+                        "peak_source": peaks["source"], "algorithmic_bytes": gu_bytes,
+                        "down_kernel": {"achieved": dn_bytes / (dn_ms * 1e-3) / 1e9,
+                                        "frac": dn_bytes / (dn_ms * 1e-3) / 1e9 / peaks["hbm"]},
+                        "whole_step_frac": (gu_bytes + dn_bytes) / (ms_step * 1e-3) / 1e9 / peaks["hbm"]}
+        else:
+            gu_flop = pairs * 4 * H * F
+            dn_flop = pairs * 2 * H * F
+            ach = gu_flop / (gu_ms * 1e-3) / 1e12
+            roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel<gate_up>", "achieved": ach,
+                        "peak": peaks["tf_sust"], "unit": "TFLOP/s", "frac": ach / peaks["tf_sust"],
+                        "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)",
+                        "frac_of_burst": ach / peaks["tf_burst"],
+                        "down_kernel": {"achieved": dn_flop / (dn_ms * 1e-3) / 1e12,
+                                        "frac": dn_flop / (dn_ms * 1e-3) / 1e12 / peaks["tf_sust"]},
+                        "whole_step_frac": (gu_flop + dn_flop) / (ms_step * 1e-3) / 1e12 / peaks["tf_sust"]}
+    elif a.workload == "search":
+        flop = 98 * 0 + 2 * (6 * T * E * H * F)  # two searches, each one all-experts GEMM pass
+        ach = flop / (ms_step * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel (all experts, whole search step)",
+                    "achieved": ach, "peak": peaks["tf_sust"], "unit": "TFLOP/s",
+                    "frac": ach / peaks["tf_sust"], "traffic": None,
+                    "peak_source": peaks["source"] + " (sustained bf16)"}
+
+    # oracle on the host cores, bounded sample (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not a.no_cpu_baseline:
+        from oracle import moe_oracle as O
+        b = synth.bf16_bits
+        Wh = dict(Wg=b(W.W_gate), W1=b(W.W1), W3=b(W.W3), W2=b(W.W2))
+        xhb = b(x)
+        n_sample = min(T, a.ref_sample if a.workload != "search" else max(4, a.ref_sample // 16))
+        dt = oracle_sample(a, Wh, xhb, beta, n_sample)
+        per_unit = 98 if a.workload == "search" else 1
+        cpu = {"value": n_sample * per_unit / dt, "unit": metric_unit(a)[1], "cores": O.num_threads(),
+               "kind": "oracle", "sample": "%d of %d tokens, one pass, %.1f s" % (n_sample, T, dt)}
+
+    if rank == 0:
+        metric, unit = metric_unit(a)
+        gpu_launches = launches_per_step * a.steps if launches_per_step else None
+        if a.workload == "search":
+            chunks = (T + 8191) // 8192
+            gpu_launches = a.steps * 2 * (1 + chunks * 3 + 2)
+        line = {
+            "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": a.steps,
+            "warmup": max(a.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(a), "h": H, "f": F, "E": E, "tokens": T,
+                       "kept_mask": kept, "beta": beta, "pairs": pairs, "experts_touched": touched,
+                       "parallelism": "replicas x%d, no collective" % world,
+                       "l2": "per step the kernels stream %.2f GB of weights, far above the 126 MB L2"
+                             % (touched * 3 * H * F * 2 / 1e9) if a.workload != "search" else
+                             "inputs and intermediates are GBs, far above the 126 MB L2"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "roofline": roofline,
+            "cpu_baseline": cpu, "stages": stages,
+        }
+        print(json.dumps(line), flush=True)
+    layer.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "search"])
+    ap.add_argument("--tokens", type=int, default=None)
+    ap.add_argument("--beta", default="0", choices=["0", "calibrated"])
+    ap.add_argument("--kept", default="full", choices=list(KEPT))
+    ap.add_argument("--search-r", default="6+4")
+    ap.add_argument("--ref-sample", type=int, default=64)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    a = ap.parse_args()
+    if a.tokens is None:
+        a.tokens = {"decode": 128, "prefill": 8192, "search": 32768}[a.workload]
+    if a.steps is None:
+        a.steps = {"decode": 200, "prefill": 50, "search": 5}[a.workload] if a.impl == "ours" else 5
+    if a.impl == "reference":
+        return run_reference(a)
+    return run_ours(a)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

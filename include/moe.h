@@ -157,6 +157,23 @@ int moe_rmsnorm(const void* x, int T, int h, float eps, void* out, void* cuda_st
 int moe_stack_forward(moe_layer_t* const* layers, int n_layers, const void* x, int T,
                       const float* betas, float eps, void* y);
 
+/*
+ * Per-stage device time of moe_forward, for benchmarks.  While enabled, every
+ * forward call on the handle records CUDA events on its stream at the stage
+ * boundaries (not part of the paper's method; a few microseconds per call):
+ *   stage 0  router + permutation (Sec. 3.1-3.3 routing, gather of routed rows)
+ *   stage 1  gate/up grouped GEMM with the SwiGLU epilogue
+ *   stage 2  down-projection grouped GEMM
+ *   stage 3  combine (Eq. 2)
+ * moe_profile_read synchronises the stream, writes the milliseconds summed over
+ * the calls recorded since the last enable/read into stage_ms[MOE_PROFILE_STAGES]
+ * and their number into *calls (host memory), and starts a new window.  At most
+ * 8192 calls are recorded per window.
+ */
+#define MOE_PROFILE_STAGES 4
+int moe_profile_enable(moe_layer_t* layer, int on);
+int moe_profile_read(moe_layer_t* layer, float* stage_ms, int* calls);
+
 /* 0 when no kernel of this handle has reported a bounded wait expiring since
  * the last call of this function, else MOE_ERR_DEVICE_TIMEOUT.  Synchronises. */
 int moe_device_status(moe_layer_t* layer);

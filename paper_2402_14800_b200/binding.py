@@ -65,6 +65,8 @@ def load_library(path: str | None = None):
     lib.moe_rmsnorm.argtypes = [vp, ci, ci, cf, vp, vp]
     lib.moe_stack_forward.argtypes = [ctypes.POINTER(vp), ci, vp, ci, ctypes.POINTER(cf), cf, vp]
     lib.moe_device_status.argtypes = [vp]
+    lib.moe_profile_enable.argtypes = [vp, ci]
+    lib.moe_profile_read.argtypes = [vp, ctypes.POINTER(cf), ctypes.POINTER(ci)]
     lib.moe_last_error.restype = ctypes.c_char_p
     if path is None:
         _lib = lib
@@ -196,6 +198,16 @@ class MoeLayer:
         best = ctypes.c_uint32(0)
         _check(load_library().moe_prune_search(self._h, x_calib.data_ptr(), T, r, losses, ctypes.byref(best)))
         return list(losses)[:n], int(best.value)
+
+    def profile_enable(self, on: bool = True):
+        _check(load_library().moe_profile_enable(self._h, int(bool(on))))
+
+    def profile_read(self):
+        """Returns (stage_ms[4] summed over the recorded calls, number of calls)."""
+        ms = (ctypes.c_float * 4)()
+        n = ctypes.c_int(0)
+        _check(load_library().moe_profile_read(self._h, ms, ctypes.byref(n)))
+        return [float(v) for v in ms], int(n.value)
 
     def device_status(self) -> int:
         return int(load_library().moe_device_status(self._h))

@@ -81,6 +81,10 @@ struct moe_layer {
   CUtensorMap w13_256, w13_128, w2_256, w2_128;
   Workspace own;
   Workspace* ws = &own;
+  // per-stage device timing (off unless moe_profile_enable)
+  bool prof = false;
+  std::vector<cudaEvent_t> prof_ev;  // MOE_PROFILE_STAGES + 1 marks per recorded call
+  size_t prof_used = 0;
 };
 
 namespace {
@@ -178,6 +182,18 @@ int ensure_gemm(moe_layer* L, int T) {
   return MOE_OK;
 }
 
+// Records a stage boundary on the handle's stream while profiling is on.
+void mark(moe_layer* L) {
+  if (!L->prof) return;
+  if (L->prof_used == L->prof_ev.size()) {
+    if (L->prof_ev.size() >= 5 * 8192) return;  // enough samples; stop recording
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return;
+    L->prof_ev.push_back(e);
+  }
+  cudaEventRecord(L->prof_ev[L->prof_used++], L->stream);
+}
+
 int check_status(moe_layer* L) {
   int st = 0;
   CUDA_TRY(cudaMemcpyAsync(&st, L->ws->status.p, 4, cudaMemcpyDeviceToHost, L->stream));
@@ -200,12 +216,15 @@ int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmM
   gu.status = (int*)L->ws->status.p; dn.status = (int*)L->ws->status.p;
   if (L->debug_simt) {
     CUDA_TRY(launch_simt_gate_up(gu_A, L->W13, gu, simt_rows, L->stream));
+    mark(L);
     CUDA_TRY(launch_simt_down(dn_A, L->W2, dn, simt_rows, dn_kind, L->stream));
   } else if (weights_m) {
     CUDA_TRY(launch_gemm_weights_m(true, m_gu, gu, (L->h + 63) / 64, L->stream));
+    mark(L);
     CUDA_TRY(launch_gemm_weights_m(false, m_dn, dn, kDecodeKbPerItem, L->stream));
   } else {
     CUDA_TRY(launch_gemm_tokens_m(true, kOutActBf16, m_gu, gu, L->stream));
+    mark(L);
     CUDA_TRY(launch_gemm_tokens_m(false, dn_kind, m_dn, dn, L->stream));
   }
   return MOE_OK;
@@ -243,6 +262,8 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
     s_count = (int32_t*)(s + off[4]); s_nsk = (int32_t*)(s + off[5]); s_nt = (int32_t*)(s + off[6]);
   }
   Meta* meta = (Meta*)L->ws->meta.p;
+  if (L->prof && (L->prof_used % (MOE_PROFILE_STAGES + 1)) != 0) L->prof_used = 0;
+  mark(L);
   CUDA_TRY(launch_router((const bf16*)x, L->Wg, T, L->h, L->r, beta, L->kept, ro, st));
   CUDA_TRY(launch_scan(ro.blk_hist, nblk, L->r, dec ? 16 : kTileRows, (int32_t*)L->ws->blk_base.p, meta,
                        s_count, s_nsk, s_nt, L->kept, L->E, st));
@@ -251,6 +272,7 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
                           (int32_t*)L->ws->pair_pos.p, (int32_t*)L->ws->row_token.p, st));
   CUDA_TRY(launch_gather((const bf16*)x, (int32_t*)L->ws->row_token.p, meta, L->h, rows_cap,
                          (bf16*)L->ws->xperm.p, st));
+  mark(L);
 
   GemmArgs gu, dn;
   memset(&gu, 0, sizeof(gu));
@@ -269,8 +291,10 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   rc = run_expert_gemms(L, meta, wm, m_gu, m_dn, gu, dn, kOutF32, (const bf16*)L->ws->xperm.p,
                         (const bf16*)L->ws->act.p, rows_cap);
   if (rc) return rc;
+  mark(L);
   CUDA_TRY(launch_combine((const float*)L->ws->O.p, ksplit, split_stride, (int32_t*)L->ws->pair_pos.p,
                           (float*)L->ws->wn.p, (const bf16*)residual, T, L->h, (bf16*)y, st));
+  mark(L);
   return MOE_OK;
 }
 
@@ -390,6 +414,7 @@ void moe_layer_destroy(moe_layer_t* L) {
                  &L->own.s_logits, &L->own.s_yall, &L->own.s_act, &L->own.s_subsets, &L->own.s_partial, &L->own.s_loss_sq,
                  &L->own.s_losses, &L->own.s_xpad, &L->own.s_meta, &L->own.hx, &L->own.hy, &L->own.xn};
   for (Buf* b : bufs) release(L, *b);
+  for (cudaEvent_t e : L->prof_ev) cudaEventDestroy(e);
   if (L->Wg) cudaFree(L->Wg);
   if (L->W13) cudaFree(L->W13);
   if (L->W2) cudaFree(L->W2);
@@ -519,6 +544,8 @@ int moe_prune_search(moe_layer_t* L, const void* x_calib, int T, int r, float* l
   ro.skipped = (uint8_t*)L->ws->skipped.p; ro.logits = (float*)L->ws->s_logits.p;
   CUDA_TRY(launch_router((const bf16*)x_calib, L->Wg, T, h, E, 0.f, L->kept, ro, st));
   Meta* meta = (Meta*)L->ws->s_meta.p;
+  const bool prof_saved = L->prof;
+  L->prof = false;  // stage marks describe moe_forward only
   for (int t0 = 0; t0 < T; t0 += Tc) {
     const int rows = (T - t0) < Tc ? (T - t0) : Tc;
     CUDA_TRY(launch_set_dense_meta(meta, E, rows, Tc_pad, st));
@@ -529,9 +556,12 @@ int moe_prune_search(moe_layer_t* L, const void* x_calib, int T, int r, float* l
     dn.a_off_mul = 1; dn.out_row_base = t0; dn.out_off_mul = 0; dn.out_col_mul = h;
     dn.out_ld = (long long)E * h; dn.out = L->ws->s_yall.p;
     if ((rc = run_expert_gemms(L, meta, false, m_gu, m_dn, gu, dn, kOutBf16, xa,
-                               (const bf16*)L->ws->s_act.p, rows)))
+                               (const bf16*)L->ws->s_act.p, rows))) {
+      L->prof = prof_saved;
       return rc;
+    }
   }
+  L->prof = prof_saved;
   CUDA_TRY(launch_enumerate((const float*)L->ws->s_logits.p, (const bf16*)L->ws->s_yall.p, T, E, r, h,
                             (const uint32_t*)L->ws->s_subsets.p, (int)nC, (float*)L->ws->s_partial.p,
                             (double*)L->ws->s_loss_sq.p, (float*)L->ws->s_losses.p, st));
@@ -581,6 +611,30 @@ int moe_stack_forward(moe_layer_t* const* layers, int n_layers, const void* x, i
     if (rc) return rc;
     cur = y;
   }
+  return MOE_OK;
+}
+
+int moe_profile_enable(moe_layer_t* L, int on) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  L->prof = on != 0;
+  L->prof_used = 0;
+  return MOE_OK;
+}
+
+int moe_profile_read(moe_layer_t* L, float* stage_ms, int* calls) {
+  if (!L || !stage_ms || !calls) return fail(MOE_ERR_INVALID_ARG, "NULL argument");
+  CUDA_TRY(cudaStreamSynchronize(L->stream));
+  const size_t per = MOE_PROFILE_STAGES + 1;
+  const size_t n = L->prof_used / per;
+  for (int s = 0; s < MOE_PROFILE_STAGES; ++s) stage_ms[s] = 0.f;
+  for (size_t c = 0; c < n; ++c)
+    for (int s = 0; s < MOE_PROFILE_STAGES; ++s) {
+      float ms = 0.f;
+      CUDA_TRY(cudaEventElapsedTime(&ms, L->prof_ev[c * per + s], L->prof_ev[c * per + s + 1]));
+      stage_ms[s] += ms;
+    }
+  *calls = (int)n;
+  L->prof_used = 0;
   return MOE_OK;
 }
 

@@ -1,0 +1,126 @@
+"""GPU parity at the Mixtral-8x7B layer shape (h=4096, f=14336, E=8), in the launch
+configurations the benchmark times: routing on every token, outputs on sampled tokens the
+oracle computes one by one, the search on a token subsample plus invariants at full size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as O
+from paper_2402_14800_b200 import binding, build, synth
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+H, F, E = synth.MIXTRAL["h"], synth.MIXTRAL["f"], synth.MIXTRAL["E"]
+FULL = 0xFF
+DEV = "cuda:0"
+N_SAMPLE = 20
+
+
+@pytest.fixture(scope="module")
+def big():
+    build.build()
+    W = synth.make_layer_weights(H, F, E, seed=0, device=DEV)
+    b = synth.bf16_bits
+    host = dict(Wg=b(W.W_gate), W1=b(W.W1), W3=b(W.W3), W2=b(W.W2))
+    xcal = synth.make_tokens(4096, H, seed=1001, device=DEV)
+    layers = {}
+
+    def layer(kept):
+        if kept not in layers:
+            layers[kept] = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, kept)
+        return layers[kept]
+
+    yield dict(host=host, W=W, xcal=xcal, layer=layer)
+    for l in layers.values():
+        l.close()
+
+
+def calibrated_beta(big, kept):
+    got = big["layer"](kept).calibrate_beta(big["xcal"])
+    want = O.beta_median(O.route(synth.bf16_bits(big["xcal"]), big["host"]["Wg"], kept, 0.0)["ratio"])
+    assert abs(got - want) <= 2e-5 * max(1.0, want)
+    return want  # the same float goes to both sides
+
+
+def run_case(big, T, kept, beta, x_seed=1):
+    host = big["host"]
+    x = synth.make_tokens(T, H, seed=x_seed, device=DEV)
+    xb = synth.bf16_bits(x)
+    layer = big["layer"](kept)
+    stats = binding.RoutingStats(T, E, DEV)
+    y = layer.forward(x, beta, stats=stats)
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+    ora_r = O.route(xb, host["Wg"], kept, beta)
+    g_idx, g_sk = stats.idx.cpu().numpy(), stats.skipped.cpu().numpy()
+    ties, close = P.check_routing(g_idx, g_sk, stats.wn.cpu().numpy(), stats.ratio.cpu().numpy(),
+                                  ora_r, kept, beta)
+    assert ties <= max(2, T // 50) and close <= max(2, T // 200)
+    agree = (g_idx == ora_r["idx"]).all(1) & (g_sk == ora_r["skipped"])
+    rng = np.random.default_rng(T)
+    sel = np.sort(rng.choice(T, size=min(T, N_SAMPLE), replace=False))
+    ora = O.moe_forward(xb[sel], host["Wg"], host["W1"], host["W3"], host["W2"], kept, beta)
+    worst = P.check_outputs(synth.bf16_bits(y)[sel], ora["y"], agree[sel])
+    assert int(stats.n_skipped.item()) == int(g_sk.sum())
+    return worst, g_sk
+
+
+@pytest.mark.parametrize("T", [1, 8, 32, 128])
+@pytest.mark.parametrize("mode", ["beta0", "calibrated"])
+def test_decode_batches(big, T, mode):
+    beta = 0.0 if mode == "beta0" else calibrated_beta(big, FULL)
+    run_case(big, T, FULL, beta)
+
+
+@pytest.mark.parametrize("T,mode", [(2048, "beta0"), (2048, "calibrated"), (8192, "calibrated"),
+                                     (32768, "beta0"), (32768, "calibrated")])
+def test_prefill_batches(big, T, mode):
+    beta = 0.0 if mode == "beta0" else calibrated_beta(big, FULL)
+    worst, sk = run_case(big, T, FULL, beta)
+    if mode == "calibrated":
+        assert 0.4 < sk.mean() < 0.6  # the median of a separate batch skips about half
+
+
+@pytest.mark.parametrize("kept", [0x3F, 0x0F])
+@pytest.mark.parametrize("T", [16, 4096])
+def test_pruned_layers(big, kept, T):
+    beta = calibrated_beta(big, kept)
+    run_case(big, T, kept, beta)
+    per_expert = 3 * H * F * 2 + H * 2
+    assert big["layer"](kept).weight_bytes == bin(kept).count("1") * per_expert
+
+
+def test_search_subsample_matches_oracle(big):
+    host = big["host"]
+    x = synth.make_tokens(40, H, seed=1, device=DEV)
+    layer = big["layer"](FULL)
+    for r in (6, 4):
+        ora = O.prune_search_allexperts(synth.bf16_bits(x), host["Wg"], host["W1"], host["W3"], host["W2"], r)
+        losses, best = layer.prune_search(x, r)
+        P.check_search(losses, best, ora)
+
+
+def test_search_full_size_invariants(big):
+    T = 32768
+    x = synth.make_tokens(T, H, seed=1, device=DEV)
+    layer = big["layer"](FULL)
+    whole, best = layer.prune_search(x, 6)
+    again, best2 = layer.prune_search(x, 6)
+    assert whole == again and best == best2
+    assert len(whole) == 28 and min(whole) > 0 and bin(best).count("1") == 6
+    assert best == [sum(1 << i for i in c) for c in __import__("itertools").combinations(range(8), 6)][int(np.argmin(whole))]
+    a, _ = layer.prune_search(x[:10000].contiguous(), 6)
+    b, _ = layer.prune_search(x[10000:].contiguous(), 6)
+    np.testing.assert_allclose(np.square(a) + np.square(b), np.square(whole), rtol=1e-4)
+    full, bestf = layer.prune_search(x[:4096].contiguous(), 8)
+    assert full == [0.0] and bestf == FULL
+    # the loss of a subset is carried by the tokens whose top-2 it breaks: more broken tokens, on
+    # average, more loss -- checked through the routing record of the same batch
+    stats = binding.RoutingStats(T, E, DEV)
+    layer.forward(x, 0.0, stats=stats)
+    idx = stats.idx.cpu().numpy()
+    pair = (1 << idx[:, 0]) | (1 << idx[:, 1])
+    subsets = O.enumerate_subsets(8, 6)
+    broken = np.array([((pair & ~int(C)) != 0).sum() for C in subsets])
+    assert np.corrcoef(broken, np.square(whole))[0, 1] > 0.9
