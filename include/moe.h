@@ -136,6 +136,30 @@ int moe_calibrate_beta(moe_layer_t* layer, const void* x, int T, float* beta_out
 int moe_prune_search(moe_layer_t* layer, const void* x_calib, int T, int r, float* losses,
                      uint32_t* best_subset);
 
+/*
+ * moe_calibrate_beta for callers that must not allocate device memory while they
+ * run (a server whose own pool owns the whole GPU, a loop that cannot take the
+ * device-wide synchronisation of cudaMalloc).  The paper has no counterpart;
+ * the result is the same median of w_e1 / w_e0 (Sec. 3.3).
+ *   W_gate_kept [r][h] bf16 device: the router rows of the kept experts, in
+ *   ascending expert order (the whole W_gate when nothing is pruned);
+ *   x [T][h] bf16 device; stream is a cudaStream_t; *beta_out is host memory.
+ * The scratch of the two kernels (per-token routing record, 21 bytes per token)
+ * lives in a fixed array inside the library image, about 340 KB that every GPU
+ * loading the library holds until the process exits; T is therefore limited to
+ * MOE_NOALLOC_MAX_TOKENS and larger T is rejected with MOE_ERR_INVALID_ARG.
+ * The call makes no cudaMalloc/cudaFree and calls no allocating library
+ * routine.  Its first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress); make that first call before any stream capture.
+ * All calls share the one array, which keeps the previous call's contents:
+ * every element that is read is rewritten first, so nothing needs clearing,
+ * but two calls that overlap on the GPU (different streams or threads) race.
+ * Synchronises the stream.
+ */
+#define MOE_NOALLOC_MAX_TOKENS 16384
+int moe_calibrate_beta_noalloc(const void* W_gate_kept, const void* x, int T, int h, int r,
+                               void* cuda_stream, float* beta_out);
+
 /* Number of subsets moe_prune_search scores: C(E, r), 0 if out of range. */
 long moe_num_subsets(int E, int r);
 

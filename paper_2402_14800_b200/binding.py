@@ -67,6 +67,7 @@ def load_library(path: str | None = None):
     lib.moe_device_status.argtypes = [vp]
     lib.moe_profile_enable.argtypes = [vp, ci]
     lib.moe_profile_read.argtypes = [vp, ctypes.POINTER(cf), ctypes.POINTER(ci)]
+    lib.moe_calibrate_beta_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, ctypes.POINTER(cf)]
     lib.moe_last_error.restype = ctypes.c_char_p
     if path is None:
         _lib = lib
@@ -211,6 +212,21 @@ class MoeLayer:
 
     def device_status(self) -> int:
         return int(load_library().moe_device_status(self._h))
+
+
+def calibrate_beta_noalloc(W_gate_kept, x, stream=None) -> float:
+    """``moe_calibrate_beta_noalloc``: the beta median without any device allocation by the
+    library (scratch is a fixed array inside it; at most 16384 tokens).  ``W_gate_kept`` holds
+    the router rows of the kept experts, ``x`` the calibration tokens."""
+    r, h = W_gate_kept.shape
+    T = x.shape[0]
+    _dev_bf16(W_gate_kept)
+    _dev_bf16(x, (T, h))
+    st = stream or torch.cuda.current_stream(x.device)
+    out = ctypes.c_float(0)
+    _check(load_library().moe_calibrate_beta_noalloc(W_gate_kept.data_ptr(), x.data_ptr(), T, h, r,
+                                                     ctypes.c_void_p(st.cuda_stream), ctypes.byref(out)))
+    return float(out.value)
 
 
 def rmsnorm(x, eps: float = 1e-5, out=None, stream=None):

@@ -68,6 +68,14 @@ struct Workspace {
   Buf hx, hy, xn;
 };
 
+int moe::set_error(int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
 struct moe_layer {
   int h = 0, f = 0, E = 0, r = 0;
   uint32_t kept_mask = 0;

@@ -37,6 +37,9 @@ struct KeptIds {
   int32_t id[kMaxE];  // compact index -> original expert id
 };
 
+// Stores the message moe_last_error() returns on this thread and returns `code` (api.cu).
+int set_error(int code, const char* fmt, ...);
+
 // ---- routing / permutation / element-wise kernels (route_permute.cu) --------------------
 struct RouteOut {
   int32_t* idx;       // [T][2] compact expert index
