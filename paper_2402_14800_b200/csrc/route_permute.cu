@@ -29,6 +29,180 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 
 // ------------------------------------------------------------------------------- router
 
+// Routing decision of one token from its r logits (one thread); writes the per-token record.
+template <int R>
+__device__ __forceinline__ void route_decide(const float (&acc)[R], int r, float beta, int t,
+                                             const KeptIds& kept, const RouteOut& o, int& e0,
+                                             int& e1, bool& skip) {
+  // top-2 on the logits (softmax is increasing), ties to the lower index
+  e0 = 0;
+  float l0 = acc[0];
+#pragma unroll
+  for (int c = 1; c < R; ++c)
+    if (c < r && acc[c] > l0) { l0 = acc[c]; e0 = c; }
+  e1 = -1;
+  float l1 = 0.f;
+#pragma unroll
+  for (int c = 0; c < R; ++c)
+    if (c < r && c != e0 && (e1 < 0 || acc[c] > l1)) { l1 = acc[c]; e1 = c; }
+  // softmax numerators relative to the maximum: p_e0 = 1, p_e1 = exp(l1 - l0); the
+  // denominator cancels in the ratio, the skip test and the normalised weights
+  const float p1 = expf(l1 - l0);
+  skip = p1 < beta * 1.0f;
+  float w0, w1;
+  if (skip) { w0 = 1.f; w1 = 0.f; }
+  else { const float d = 1.0f + p1; w0 = 1.0f / d; w1 = p1 / d; }
+  o.idx[2 * t] = e0; o.idx[2 * t + 1] = e1;
+  o.wn[2 * t] = w0; o.wn[2 * t + 1] = w1;
+  o.ratio[t] = p1;
+  o.skipped[t] = skip ? 1 : 0;
+  if (o.s_idx) {
+    o.s_idx[2 * t] = kept.id[e0]; o.s_idx[2 * t + 1] = kept.id[e1];
+    o.s_wn[2 * t] = w0; o.s_wn[2 * t + 1] = w1;
+    o.s_ratio[t] = p1;
+    o.s_skipped[t] = skip ? 1 : 0;
+  }
+  if (o.logits) {
+#pragma unroll
+    for (int c = 0; c < R; ++c)
+      if (c < r) o.logits[(size_t)t * r + c] = acc[c];
+  }
+}
+
+// Small batches: one block per token, all loads of a thread independent of each other, so the
+// kernel costs a couple of memory round trips instead of a serial walk over the row.
+template <int R>
+__global__ void __launch_bounds__(256)
+router_small_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, int h, int r,
+                    float beta, KeptIds kept, RouteOut o) {
+  __shared__ float s_part[8][R];
+  const int t = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nvec = h >> 3;
+  float acc[R];
+#pragma unroll
+  for (int c = 0; c < R; ++c) acc[c] = 0.f;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)t * h);
+  for (int v = threadIdx.x; v < nvec; v += 256) {
+    float xf[8];
+    unpack8(__ldg(xr + v), xf);
+#pragma unroll
+    for (int c = 0; c < R; ++c) {
+      if (c < r) {
+        float wf[8];
+        unpack8(__ldg(reinterpret_cast<const uint4*>(Wg + (size_t)c * h) + v), wf);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[c] = fmaf(xf[k], wf[k], acc[c]);
+      }
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < R; ++c) {
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], s);
+    if (lane == 0) s_part[warp][c] = acc[c];
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float l[R];
+#pragma unroll
+    for (int c = 0; c < R; ++c) {
+      float v = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) v += s_part[w][c];
+      l[c] = v;
+    }
+    int e0, e1;
+    bool skip;
+    route_decide<R>(l, r, beta, t, kept, o, e0, e1, skip);
+  }
+}
+
+// Small batches: the whole permutation in one block (histogram, offsets, ranks, scatter and
+// the padding rows), T <= blockDim.x.
+__global__ void __launch_bounds__(kDecodeMaxT)
+permute_small_kernel(const int32_t* __restrict__ idx, const uint8_t* __restrict__ skipped, int T,
+                     int r, int pad, Meta* meta, int32_t* __restrict__ pair_pos,
+                     int32_t* __restrict__ row_token, int32_t* s_count, int32_t* s_nskipped,
+                     int32_t* s_ntouched, KeptIds kept, int E) {
+  __shared__ int s_e[kDecodeMaxT][2];
+  __shared__ int s_cnt[kMaxE][2];
+  __shared__ int s_off[kMaxE + 1];
+  __shared__ int s_nsk;
+  const int t = threadIdx.x;
+  int e0 = -1, e1 = -1;
+  if (t < T) {
+    e0 = idx[2 * t];
+    e1 = skipped[t] ? -1 : idx[2 * t + 1];
+  }
+  s_e[t][0] = e0;
+  s_e[t][1] = e1;
+  __syncthreads();
+  if (t < 2 * r) {
+    const int c = t >> 1, slot = t & 1;
+    int n = 0;
+    for (int i = 0; i < T; ++i) n += (s_e[i][slot] == c);
+    s_cnt[c][slot] = n;
+  } else if (t == 2 * kMaxE) {
+    int n = 0;
+    for (int i = 0; i < T; ++i) n += (s_e[i][1] < 0);
+    s_nsk = n;
+  }
+  __syncthreads();
+  if (t == 0) {
+    int off = 0, tiles = 0, touched = 0;
+    meta->off[0] = 0;
+    meta->tile_prefix[0] = 0;
+    s_off[0] = 0;
+    for (int c = 0; c < kMaxE; ++c) {
+      const int n0 = c < r ? s_cnt[c][0] : 0, n1 = c < r ? s_cnt[c][1] : 0;
+      const int n = n0 + n1;
+      meta->count[c] = n;
+      meta->count_slot[c][0] = n0;
+      meta->count_slot[c][1] = n1;
+      off += (n + pad - 1) / pad * pad;
+      tiles += (n + kTileRows - 1) / kTileRows;
+      touched += (n > 0);
+      meta->off[c + 1] = off;
+      meta->tile_prefix[c + 1] = tiles;
+      s_off[c + 1] = off;
+    }
+    meta->rows_total = off;
+    meta->n_skipped = s_nsk;
+    meta->n_touched = touched;
+    meta->reserved = 0;
+    if (s_count) {
+      for (int e = 0; e < E; ++e) { s_count[2 * e] = 0; s_count[2 * e + 1] = 0; }
+      for (int c = 0; c < r; ++c) {
+        s_count[2 * kept.id[c]] = s_cnt[c][0];
+        s_count[2 * kept.id[c] + 1] = s_cnt[c][1];
+      }
+      *s_nskipped = s_nsk;
+      *s_ntouched = touched;
+    }
+  }
+  __syncthreads();
+  if (t < T) {
+    int r0 = 0, r1 = 0;
+    for (int i = 0; i < t; ++i) {
+      r0 += (s_e[i][0] == e0) + (s_e[i][1] == e0);
+      r1 += (s_e[i][0] == e1) + (s_e[i][1] == e1);
+    }
+    const int p0 = s_off[e0] + r0;
+    row_token[p0] = t;
+    pair_pos[2 * t] = p0;
+    int p1 = -1;
+    if (e1 >= 0) {
+      p1 = s_off[e1] + r1;
+      row_token[p1] = t;
+    }
+    pair_pos[2 * t + 1] = p1;
+  }
+  if (t < r) {  // padding rows of this expert's group gather zeros
+    for (int row = s_off[t] + s_cnt[t][0] + s_cnt[t][1]; row < s_off[t + 1]; ++row) row_token[row] = -1;
+  }
+}
+
 template <int R>
 __global__ void __launch_bounds__(256)
 router_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, int h, int r,
@@ -69,39 +243,9 @@ router_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, in
       for (int s = 16; s > 0; s >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], s);
     }
     if (lane == 0) {
-      // top-2 on the logits (softmax is increasing), ties to the lower index
-      int e0 = 0;
-      float l0 = acc[0];
-#pragma unroll
-      for (int c = 1; c < R; ++c)
-        if (c < r && acc[c] > l0) { l0 = acc[c]; e0 = c; }
-      int e1 = -1;
-      float l1 = 0.f;
-#pragma unroll
-      for (int c = 0; c < R; ++c)
-        if (c < r && c != e0 && (e1 < 0 || acc[c] > l1)) { l1 = acc[c]; e1 = c; }
-      // softmax numerators relative to the maximum: p_e0 = 1, p_e1 = exp(l1 - l0); the
-      // denominator cancels in the ratio, the skip test and the normalised weights
-      const float p1 = expf(l1 - l0);
-      const bool skip = p1 < beta * 1.0f;
-      float w0, w1;
-      if (skip) { w0 = 1.f; w1 = 0.f; }
-      else { const float d = 1.0f + p1; w0 = 1.0f / d; w1 = p1 / d; }
-      o.idx[2 * t] = e0; o.idx[2 * t + 1] = e1;
-      o.wn[2 * t] = w0; o.wn[2 * t + 1] = w1;
-      o.ratio[t] = p1;
-      o.skipped[t] = skip ? 1 : 0;
-      if (o.s_idx) {
-        o.s_idx[2 * t] = kept.id[e0]; o.s_idx[2 * t + 1] = kept.id[e1];
-        o.s_wn[2 * t] = w0; o.s_wn[2 * t + 1] = w1;
-        o.s_ratio[t] = p1;
-        o.s_skipped[t] = skip ? 1 : 0;
-      }
-      if (o.logits) {
-#pragma unroll
-        for (int c = 0; c < R; ++c)
-          if (c < r) o.logits[(size_t)t * r + c] = acc[c];
-      }
+      int e0, e1;
+      bool skip;
+      route_decide<R>(acc, r, beta, t, kept, o, e0, e1, skip);
       s_e[tl][0] = e0;
       s_e[tl][1] = skip ? -1 : e1;
       s_skip[tl] = skip ? 1 : 0;
@@ -424,6 +568,27 @@ cudaError_t launch_router(const bf16* x, const bf16* Wg, int T, int h, int r, fl
     case 7: case 8: router_kernel<8><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
     default: router_kernel<kMaxE><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_router_small(const bf16* x, const bf16* Wg, int T, int h, int r, float beta,
+                                const KeptIds& kept, const RouteOut& out, cudaStream_t st) {
+  switch (r) {
+    case 2: router_small_kernel<2><<<T, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+    case 3: case 4: router_small_kernel<4><<<T, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+    case 5: case 6: router_small_kernel<6><<<T, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+    case 7: case 8: router_small_kernel<8><<<T, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+    default: router_small_kernel<kMaxE><<<T, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_permute_small(const int32_t* idx, const uint8_t* skipped, int T, int r, int pad,
+                                 Meta* meta, int32_t* pair_pos, int32_t* row_token,
+                                 int32_t* s_count, int32_t* s_nskipped, int32_t* s_ntouched,
+                                 const KeptIds& kept, int E, cudaStream_t st) {
+  permute_small_kernel<<<1, kDecodeMaxT, 0, st>>>(idx, skipped, T, r, pad, meta, pair_pos, row_token,
+                                                  s_count, s_nskipped, s_ntouched, kept, E);
   return cudaGetLastError();
 }
 
