@@ -135,10 +135,54 @@ def host_inputs(a, device):
     return W, x, xcal
 
 
+def run_reference_stack(a):
+    """Oracle over the first layers of the stack (each layer's weights are 2.8 GB on the host, so
+    only min(layers, 4) layers are walked; the sample line says so)."""
+    from oracle import moe_oracle as O
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    b = synth.bf16_bits
+    nl = min(a.layers, 4)
+    n_sample = max(1, min(a.tokens, 8))
+    xh = b(synth.make_tokens(a.tokens, H, seed=1, device=dev))[:n_sample]
+    Ws = []
+    for l in range(nl):
+        W = synth.make_layer_weights(H, F, E, seed=100 + l, device=dev)
+        Ws.append(dict(Wg=b(W.W_gate), W1=b(W.W1), W3=b(W.W3), W2=b(W.W2)))
+        del W
+    times = []
+    for _ in range(a.steps):
+        t0 = time.perf_counter()
+        cur = xh
+        for Wh in Ws:
+            xn = O.rmsnorm(cur, 1e-5)
+            cur = O.moe_forward(xn, Wh["Wg"], Wh["W1"], Wh["W3"], Wh["W2"], 0xFF, 0.0, residual=cur)["y"]
+        times.append(time.perf_counter() - t0)
+    # tokens/s through a 32-layer stack, extrapolated linearly from the layers walked
+    value = n_sample * a.steps / (sum(times) * a.layers / nl)
+    sample = "%d of %d tokens through %d of %d layers per step, scaled to all layers" % (
+        n_sample, a.tokens, nl, a.layers)
+    line = {
+        "impl": "reference",
+        "metric": "MoE-stack tokens/s on 1 B200 (32 layers, RMSNorm + residual, attention omitted)",
+        "value": value, "unit": "tokens/s", "n_gpus": a.gpus, "steps": a.steps, "warmup": a.warmup,
+        "ms_per_step": 1e3 * sum(times) / a.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "stack%d_T%d_full_beta-0" % (a.layers, a.tokens), "h": H, "f": F, "E": E},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": O.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def run_reference(a):
     rank, world, local = dist_env()
     if rank != 0:
         return 0
+    if a.workload == "stack":
+        return run_reference_stack(a)
     from oracle import moe_oracle as O
     dev = "cuda:0" if torch.cuda.is_available() else "cpu"
     W, x, xcal = host_inputs(a, dev)
@@ -364,13 +408,171 @@ def run_ours(a):
     return 0
 
 
+# ----------------------------------------------------------------- stack of 32 layers
+
+def run_stack(a):
+    """x_{l+1} = x_l + MoE_l(RMSNorm(x_l)) over `--layers` Mixtral-shaped layers (attention left
+    out), each layer with its own seed.  Pruned variants take each layer's kept subset from the
+    layer-wise search on calibration states of the unpruned stack; beta is calibrated per layer."""
+    from paper_2402_14800_b200 import binding, build
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (sm_100a); there is no CPU fallback")
+    build.build()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = measured_peaks()
+    T, NL = a.tokens, a.layers
+    r = {"full": 8, "r6": 6, "r4": 4}[a.kept]
+    x = synth.make_tokens(T, H, seed=1, device=dev)
+    state = synth.make_tokens(a.cal_tokens, H, seed=1001, device=dev)
+    layers, betas, masks, search_ms = [], [], [], 0.0
+    for l in range(NL):
+        W = synth.make_layer_weights(H, F, E, seed=100 + l, device=dev)
+        xn = binding.rmsnorm(state)
+        if r == 8:
+            layer = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, 0xFF)
+            if layers:
+                layer.share_scratch(layers[0])
+            state = layer.forward(xn, 0.0, residual=state)
+            mask = 0xFF
+        else:
+            full = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, 0xFF)
+            torch.cuda.synchronize(dev)
+            t0 = time.perf_counter()
+            _, mask = full.prune_search(xn, r)
+            search_ms += 1e3 * (time.perf_counter() - t0)
+            state = full.forward(xn, 0.0, residual=state)
+            torch.cuda.synchronize(dev)
+            full.close()
+            layer = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, mask)
+            if layers:
+                layer.share_scratch(layers[0])
+        betas.append(layer.calibrate_beta(xn) if a.beta == "calibrated" else 0.0)
+        masks.append(mask)
+        layers.append(layer)
+        del W
+    del state, xn
+    stream = torch.cuda.Stream(dev)
+    for layer in layers:
+        layer.set_stream(stream)
+    weight_bytes = sum(l.weight_bytes for l in layers)
+    y = torch.empty_like(x)
+
+    # routing facts per layer (untimed): experts touched and pairs, along the real trajectory
+    touched, pairs = [], []
+    with torch.cuda.stream(stream):
+        cur = x
+        stats = binding.RoutingStats(T, E, dev)
+        for layer, b in zip(layers, betas):
+            xn = binding.rmsnorm(cur, stream=stream)
+            cur = layer.forward(xn, b, residual=cur, stats=stats)
+            stream.synchronize()
+            touched.append(int(stats.n_experts_touched.item()))
+            pairs.append(2 * T - int(stats.n_skipped.item()))
+
+    def step():
+        binding.stack_forward(layers, x, betas, 1e-5, y)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(a.warmup, 3)):
+            step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with torch.cuda.stream(stream):
+        ev0.record(stream)
+        for _ in range(a.steps):
+            step()
+        ev1.record(stream)
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / a.steps
+    value = world * T * a.steps / (ms_total * 1e-3)
+
+    xh = x.cpu().pin_memory()
+    yh = torch.empty_like(xh).pin_memory()
+    xd = torch.empty_like(x)
+    n_e2e = max(3, min(a.steps, 20))
+    barrier()
+    t0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        for _ in range(n_e2e):
+            xd.copy_(xh, non_blocking=True)
+            binding.stack_forward(layers, xd, betas, 1e-5, y)
+            yh.copy_(y, non_blocking=True)
+            stream.synchronize()
+    dt = time.perf_counter() - t0
+    e2e = {"value": world * T * n_e2e / dt, "unit": "tokens/s", "h2d_bytes_per_step": T * H * 2,
+           "d2h_bytes_per_step": T * H * 2,
+           "timing": "host wall clock; pinned-host copies around moe_stack_forward on one stream"}
+
+    if T <= 256:
+        nbytes = sum(touched) * 3 * H * F * 2
+        ach = nbytes / (ms_step * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "whole stack step (weight-major GEMMs dominate)",
+                    "achieved": ach, "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"],
+                    "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": nbytes}
+    else:
+        flop = sum(pairs) * FLOP_PER_PAIR
+        ach = flop / (ms_step * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "whole stack step (token-major GEMMs dominate)",
+                    "achieved": ach, "peak": peaks["tf_sust"], "unit": "TFLOP/s",
+                    "frac": ach / peaks["tf_sust"], "traffic": None,
+                    "peak_source": peaks["source"] + " (sustained bf16)"}
+    if rank == 0:
+        per_layer = (6 if T <= 256 else 7) + 1
+        line = {
+            "metric": "MoE-stack tokens/s on 1 B200 (32 layers, RMSNorm + residual, attention omitted)",
+            "value": value, "unit": "tokens/s", "n_gpus": world, "steps": a.steps,
+            "warmup": max(a.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "stack%d_T%d_%s_beta-%s" % (NL, T, a.kept, a.beta), "h": H, "f": F,
+                       "E": E, "tokens": T, "layers": NL, "kept_masks": masks,
+                       "betas": [round(b, 4) for b in betas], "weight_bytes": weight_bytes,
+                       "experts_touched_sum": sum(touched), "pairs_sum": sum(pairs),
+                       "search_ms_total": search_ms, "calibration_tokens": a.cal_tokens,
+                       "parallelism": "replicas x%d, no collective" % world,
+                       "l2": "each layer streams its own weights (GBs), far above the 126 MB L2"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": per_layer * NL * a.steps,
+            "roofline": roofline, "cpu_baseline": None, "stages": None,
+        }
+        print(json.dumps(line), flush=True)
+    for layer in reversed(layers):
+        layer.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "search"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "search", "stack"])
+    ap.add_argument("--layers", type=int, default=32)
+    ap.add_argument("--cal-tokens", type=int, default=4096)
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--beta", default="0", choices=["0", "calibrated"])
     ap.add_argument("--kept", default="full", choices=list(KEPT))
@@ -379,11 +581,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     a = ap.parse_args()
     if a.tokens is None:
-        a.tokens = {"decode": 128, "prefill": 8192, "search": 32768}[a.workload]
+        a.tokens = {"decode": 128, "prefill": 8192, "search": 32768, "stack": 16}[a.workload]
     if a.steps is None:
-        a.steps = {"decode": 200, "prefill": 50, "search": 5}[a.workload] if a.impl == "ours" else 5
+        a.steps = {"decode": 200, "prefill": 50, "search": 5, "stack": 10}[a.workload] if a.impl == "ours" else 5
     if a.impl == "reference":
         return run_reference(a)
+    if a.workload == "stack":
+        return run_stack(a)
     return run_ours(a)
 
 

@@ -63,6 +63,14 @@ void moe_layer_destroy(moe_layer_t* layer);
 /* Stream (a cudaStream_t) that later calls on this handle enqueue on. */
 int moe_set_stream(moe_layer_t* layer, void* cuda_stream);
 
+/*
+ * Let `layer` run out of `owner`'s scratch buffers instead of its own (a stack of
+ * layers then needs one set of scratch, not one per layer).  Both must have the
+ * same h and f and must never run at the same time; `owner` must outlive the
+ * sharing.  owner == NULL returns `layer` to its own scratch.
+ */
+int moe_layer_share_scratch(moe_layer_t* layer, moe_layer_t* owner);
+
 /* Bytes of device memory the handle holds for weights (router + kept experts). */
 size_t moe_layer_weight_bytes(const moe_layer_t* layer);
 

@@ -65,6 +65,7 @@ def load_library(path: str | None = None):
     lib.moe_rmsnorm.argtypes = [vp, ci, ci, cf, vp, vp]
     lib.moe_stack_forward.argtypes = [ctypes.POINTER(vp), ci, vp, ci, ctypes.POINTER(cf), cf, vp]
     lib.moe_device_status.argtypes = [vp]
+    lib.moe_layer_share_scratch.argtypes = [vp, vp]
     lib.moe_profile_enable.argtypes = [vp, ci]
     lib.moe_profile_read.argtypes = [vp, ctypes.POINTER(cf), ctypes.POINTER(ci)]
     lib.moe_calibrate_beta_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, ctypes.POINTER(cf)]
@@ -149,6 +150,10 @@ class MoeLayer:
 
     def set_stream(self, stream: torch.cuda.Stream):
         _check(load_library().moe_set_stream(self._h, ctypes.c_void_p(stream.cuda_stream)))
+
+    def share_scratch(self, owner: "MoeLayer | None"):
+        """Run out of ``owner``'s scratch buffers (``moe_layer_share_scratch``)."""
+        _check(load_library().moe_layer_share_scratch(self._h, owner._h if owner is not None else None))
 
     @property
     def weight_bytes(self) -> int:

@@ -614,17 +614,32 @@ int moe_stack_forward(moe_layer_t* const* layers, int n_layers, const void* x, i
   for (int l = 0; l < n_layers; ++l) {
     moe_layer* L = layers[l];
     cudaStream_t saved = L->stream;
+    Workspace* saved_ws = L->ws;
     L->stream = L0->stream;
-    L->ws = (L->f == L0->f) ? &L0->own : &L->own;
+    if (L->f == L0->f) L->ws = L0->ws;
     rc = MOE_OK;
     cudaError_t e = launch_rmsnorm((const bf16*)cur, T, L->h, eps, (bf16*)L0->ws->xn.p, L0->stream);
     if (e != cudaSuccess) rc = fail(MOE_ERR_CUDA, "rmsnorm: %s", cudaGetErrorString(e));
     if (!rc) rc = forward_impl(L, L0->ws->xn.p, T, betas ? betas[l] : 0.f, cur, y, nullptr);
     L->stream = saved;
-    L->ws = &L->own;
+    L->ws = saved_ws;
     if (rc) return rc;
     cur = y;
   }
+  return MOE_OK;
+}
+
+int moe_layer_share_scratch(moe_layer_t* L, moe_layer_t* owner) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  if (!owner || owner == L) {
+    L->ws = &L->own;
+    return MOE_OK;
+  }
+  if (owner->h != L->h || owner->f != L->f)
+    return fail(MOE_ERR_INVALID_ARG, "scratch can only be shared between layers of the same h and f");
+  if (owner->ws != &owner->own)
+    return fail(MOE_ERR_INVALID_ARG, "the owner itself borrows its scratch");
+  L->ws = &owner->own;
   return MOE_OK;
 }
 
