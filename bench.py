@@ -42,6 +42,20 @@ def measured_peaks():
     return dict(hbm=6650.0, tf_burst=1590.0, tf_sust=1400.0, source="fallback")
 
 
+def recorded_traffic(workload: str):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu capture of this
+    workload, or None when there is none or the kernel source changed since."""
+    import hashlib
+    try:
+        rec = json.load(open(os.path.join(ROOT, "profiles", "traffic.json"))).get(workload)
+        src = os.path.join(ROOT, "paper_2402_14800_b200", "csrc", "gemm_sm100.cu")
+        if rec and hashlib.sha256(open(src, "rb").read()).hexdigest() == rec["kernel_source_sha256"]:
+            return rec["dram_bytes"]
+    except Exception:
+        pass
+    return None
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -94,6 +108,23 @@ def dist_env():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     return rank, world, local
+
+
+def max_over_ranks(v: float, dev=None) -> float:
+    """Max of a per-rank scalar over all ranks (identity for a single process)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(v)
+    on_gpu = dist.get_backend() == "nccl"
+    t = torch.tensor([v], dtype=torch.float64, device=dev if on_gpu else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank_step: float, steps: int, ms_total_max: float, world: int) -> float:
+    """Replicas: every rank processes its own units; the job's rate is all of them over the
+    slowest rank's time."""
+    return world * units_per_rank_step * steps / (ms_total_max * 1e-3)
 
 
 def workload_name(a):
@@ -296,13 +327,9 @@ def run_ours(a):
     if a.workload != "search":
         stage_ms, ncalls = layer.profile_read()
         layer.profile_enable(False)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dev)
     ms_step = ms_total / a.steps
-    value = world * units_per_step(a) * a.steps / (ms_total * 1e-3)
+    value = whole_job_value(units_per_step(a), a.steps, ms_total, world)
 
     # end to end through the host-buffer entry point (forward workloads only)
     e2e = None
@@ -318,11 +345,7 @@ def run_ours(a):
             layer.forward_host(xh, beta, yh)
         torch.cuda.synchronize(dev)
         dt = time.perf_counter() - t0
-        if world > 1:
-            import torch.distributed as dist
-            tt = torch.tensor([dt], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            dt = float(tt.item())
+        dt = max_over_ranks(dt, dev)
         e2e = {"value": world * T * n_e2e / dt, "unit": "tokens/s", "h2d_bytes_per_step": T * H * 2,
                "d2h_bytes_per_step": T * H * 2, "timing": "host wall clock around the C-ABI call, max over ranks"}
     else:
@@ -344,7 +367,8 @@ def run_ours(a):
             dn_bytes = touched * H * F * 2 + pairs * F * 2 + 7 * pairs * H * 4
             ach = gu_bytes / (gu_ms * 1e-3) / 1e9
             roofline = {"bound": "hbm", "kernel": "gemm_weights_m_kernel<gate_up>", "achieved": ach,
-                        "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"], "traffic": None,
+                        "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"],
+                        "traffic": recorded_traffic(workload_name(a)),
                         "peak_source": peaks["source"], "algorithmic_bytes": gu_bytes,
                         "down_kernel": {"achieved": dn_bytes / (dn_ms * 1e-3) / 1e9,
                                         "frac": dn_bytes / (dn_ms * 1e-3) / 1e9 / peaks["hbm"]},
@@ -355,7 +379,8 @@ def run_ours(a):
             ach = gu_flop / (gu_ms * 1e-3) / 1e12
             roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel<gate_up>", "achieved": ach,
                         "peak": peaks["tf_sust"], "unit": "TFLOP/s", "frac": ach / peaks["tf_sust"],
-                        "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)",
+                        "traffic": recorded_traffic(workload_name(a)),
+                        "peak_source": peaks["source"] + " (sustained bf16)",
                         "frac_of_burst": ach / peaks["tf_burst"],
                         "down_kernel": {"achieved": dn_flop / (dn_ms * 1e-3) / 1e12,
                                         "frac": dn_flop / (dn_ms * 1e-3) / 1e12 / peaks["tf_sust"]},
@@ -500,13 +525,9 @@ def run_stack(a):
     barrier()
     ms_total = ev0.elapsed_time(ev1)
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dev)
     ms_step = ms_total / a.steps
-    value = world * T * a.steps / (ms_total * 1e-3)
+    value = whole_job_value(T, a.steps, ms_total, world)
 
     xh = x.cpu().pin_memory()
     yh = torch.empty_like(xh).pin_memory()
