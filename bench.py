@@ -70,7 +70,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
@@ -311,8 +311,6 @@ def run_ours(a):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    if a.workload != "search":
-        layer.profile_enable(True)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     with torch.cuda.stream(stream):
@@ -322,11 +320,18 @@ def run_ours(a):
         ev1.record(stream)
     barrier()
     ms_total = ev0.elapsed_time(ev1)
-    clocks = sampler.stop() if rank == 0 else None
+    # the same K steps once more with an event at every stage boundary: per-kernel durations for
+    # the roofline.  (The events sit between the kernels, so this pass does not overlap one
+    # kernel's launch with its predecessor's tail; `value` comes from the pass above.)
     stage_ms, ncalls = ([0, 0, 0, 0], 0)
     if a.workload != "search":
+        layer.profile_enable(True)
+        with torch.cuda.stream(stream):
+            for _ in range(a.steps):
+                step()
         stage_ms, ncalls = layer.profile_read()
         layer.profile_enable(False)
+    clocks = sampler.stop() if rank == 0 else None
     ms_total = max_over_ranks(ms_total, dev)
     ms_step = ms_total / a.steps
     value = whole_job_value(units_per_step(a), a.steps, ms_total, world)
@@ -598,13 +603,13 @@ def main():
     ap.add_argument("--beta", default="0", choices=["0", "calibrated"])
     ap.add_argument("--kept", default="full", choices=list(KEPT))
     ap.add_argument("--search-r", default="6+4")
-    ap.add_argument("--ref-sample", type=int, default=64)
+    ap.add_argument("--ref-sample", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     a = ap.parse_args()
     if a.tokens is None:
         a.tokens = {"decode": 128, "prefill": 8192, "search": 32768, "stack": 16}[a.workload]
     if a.steps is None:
-        a.steps = {"decode": 200, "prefill": 50, "search": 5, "stack": 10}[a.workload] if a.impl == "ours" else 5
+        a.steps = {"decode": 2000, "prefill": 100, "search": 5, "stack": 10}[a.workload] if a.impl == "ours" else 5
     if a.impl == "reference":
         return run_reference(a)
     if a.workload == "stack":

@@ -37,6 +37,34 @@ struct KeptIds {
   int32_t id[kMaxE];  // compact index -> original expert id
 };
 
+// Programmatic dependent launch: a kernel launched this way may start while its predecessor
+// in the stream is still draining; it must call pdl_wait() before touching anything the
+// predecessor wrote (or still reads).  Every kernel on the forward path calls
+// pdl_launch_dependents() and pdl_wait() first thing (the GEMMs after their set-up), so the
+// stream order of all memory accesses is unchanged and only launch latency and prologues overlap.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                       Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // Stores the message moe_last_error() returns on this thread and returns `code` (api.cu).
 int set_error(int code, const char* fmt, ...);
 

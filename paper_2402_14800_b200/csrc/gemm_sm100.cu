@@ -292,13 +292,16 @@ gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args)
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
-    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
   setup_barriers<TM_NS>(bars);
   if (warp == 1) {
     tmem_alloc(smem_u32(&bars.tmem_base), 512);
     tmem_relinquish();
   }
+  // everything above is independent of the preceding kernels; their results are read from here on
+  pdl_launch_dependents();
+  pdl_wait();
+  for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
+    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -469,13 +472,16 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
-    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
   setup_barriers<WM_NS>(bars);
   if (warp == 1) {
     tmem_alloc(smem_u32(&bars.tmem_base), 256);
     tmem_relinquish();
   }
+  // everything above is independent of the preceding kernels; their results are read from here on
+  pdl_launch_dependents();
+  pdl_wait();
+  for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
+    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -723,22 +729,18 @@ cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps&
                                  const GemmArgs& a, cudaStream_t st) {
   const int grid = g_num_sms > 0 ? g_num_sms : 148;
   if (gate_up)
-    gemm_tokens_m_kernel<true, kOutActBf16><<<grid, kThreads, TM_SMEM, st>>>(maps, a);
-  else if (out_kind == kOutF32)
-    gemm_tokens_m_kernel<false, kOutF32><<<grid, kThreads, TM_SMEM, st>>>(maps, a);
-  else
-    gemm_tokens_m_kernel<false, kOutBf16><<<grid, kThreads, TM_SMEM, st>>>(maps, a);
-  return cudaGetLastError();
+    return launch_pdl(gemm_tokens_m_kernel<true, kOutActBf16>, dim3(grid), dim3(kThreads), TM_SMEM, st, maps, a);
+  if (out_kind == kOutF32)
+    return launch_pdl(gemm_tokens_m_kernel<false, kOutF32>, dim3(grid), dim3(kThreads), TM_SMEM, st, maps, a);
+  return launch_pdl(gemm_tokens_m_kernel<false, kOutBf16>, dim3(grid), dim3(kThreads), TM_SMEM, st, maps, a);
 }
 
 cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
                                   int kb_per_item, cudaStream_t st) {
   const int grid = g_num_sms > 0 ? g_num_sms : 148;
   if (gate_up)
-    gemm_weights_m_kernel<true><<<grid, kThreads, WM_SMEM, st>>>(maps, a, kb_per_item);
-  else
-    gemm_weights_m_kernel<false><<<grid, kThreads, WM_SMEM, st>>>(maps, a, kb_per_item);
-  return cudaGetLastError();
+    return launch_pdl(gemm_weights_m_kernel<true>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a, kb_per_item);
+  return launch_pdl(gemm_weights_m_kernel<false>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a, kb_per_item);
 }
 
 cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,

@@ -75,6 +75,8 @@ template <int R>
 __global__ void __launch_bounds__(256)
 router_small_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, int h, int r,
                     float beta, KeptIds kept, RouteOut o) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float s_part[8][R];
   const int t = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -125,6 +127,8 @@ permute_small_kernel(const int32_t* __restrict__ idx, const uint8_t* __restrict_
                      int r, int pad, Meta* meta, int32_t* __restrict__ pair_pos,
                      int32_t* __restrict__ row_token, int32_t* s_count, int32_t* s_nskipped,
                      int32_t* s_ntouched, KeptIds kept, int E) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int s_e[kDecodeMaxT][2];
   __shared__ int s_cnt[kMaxE][2];
   __shared__ int s_off[kMaxE + 1];
@@ -207,6 +211,8 @@ template <int R>
 __global__ void __launch_bounds__(256)
 router_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, int h, int r,
               float beta, KeptIds kept, RouteOut o) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int s_e[kRouteTokPerBlock][2];
   __shared__ int s_skip[kRouteTokPerBlock];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -273,6 +279,8 @@ __global__ void __launch_bounds__(1024)
 scan_kernel(const int32_t* __restrict__ blk_hist, int nblk, int r, int pad,
             int32_t* __restrict__ blk_base, Meta* meta, int32_t* s_count, int32_t* s_nskipped,
             int32_t* s_ntouched, KeptIds kept, int E) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int s_tot[kMaxE][2];
   __shared__ int s_skipped;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -348,6 +356,8 @@ __global__ void __launch_bounds__(2 * kRouteTokPerBlock)
 scatter_kernel(const int32_t* __restrict__ idx, const uint8_t* __restrict__ skipped,
                const int32_t* __restrict__ blk_base, const Meta* __restrict__ meta, int T,
                int32_t* __restrict__ pair_pos, int32_t* __restrict__ row_token) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int s_e[kRouteTokPerBlock][2];
   const int tl = threadIdx.x >> 1, slot = threadIdx.x & 1;
   const int t = blockIdx.x * kRouteTokPerBlock + tl;
@@ -374,6 +384,8 @@ scatter_kernel(const int32_t* __restrict__ idx, const uint8_t* __restrict__ skip
 __global__ void __launch_bounds__(256)
 gather_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ row_token,
               const Meta* __restrict__ meta, int h, bf16* __restrict__ xperm) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int rows = meta->rows_total;
   const int lane = threadIdx.x & 31;
   const int nvec = h >> 3;
@@ -395,14 +407,17 @@ __global__ void __launch_bounds__(128)
 combine_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
                const int32_t* __restrict__ pair_pos, const float* __restrict__ wn,
                const bf16* residual, int T, int h, bf16* y) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int t = blockIdx.x;
   const int p0 = pair_pos[2 * t], p1 = pair_pos[2 * t + 1];
   const float w0 = wn[2 * t], w1 = wn[2 * t + 1];
   const int nvec = h >> 3;
-  for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+  for (int v = blockIdx.y * blockDim.x + threadIdx.x; v < nvec; v += gridDim.y * blockDim.x) {
     float a[8], b[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) { a[k] = 0.f; b[k] = 0.f; }
+#pragma unroll 4
     for (int s = 0; s < ksplit; ++s) {
       const float4* o0 = reinterpret_cast<const float4*>(O + s * split_stride + (size_t)p0 * h) + 2 * v;
       const float4 q0 = o0[0], q1 = o0[1];
@@ -435,6 +450,8 @@ combine_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
 
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const bf16* x, int T, int h, float eps, bf16* out) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float s_part[8];
   const int t = blockIdx.x;
   const int nvec = h >> 3;
@@ -562,11 +579,11 @@ cudaError_t launch_router(const bf16* x, const bf16* Wg, int T, int h, int r, fl
                           const KeptIds& kept, const RouteOut& out, cudaStream_t st) {
   const int nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
   switch (r) {
-    case 2: router_kernel<2><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
-    case 3: case 4: router_kernel<4><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
-    case 5: case 6: router_kernel<6><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
-    case 7: case 8: router_kernel<8><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
-    default: router_kernel<kMaxE><<<nblk, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+    case 2: return launch_pdl(router_kernel<2>, dim3(nblk), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
+    case 3: case 4: return launch_pdl(router_kernel<4>, dim3(nblk), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
+    case 5: case 6: return launch_pdl(router_kernel<6>, dim3(nblk), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
+    case 7: case 8: return launch_pdl(router_kernel<8>, dim3(nblk), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
+    default: return launch_pdl(router_kernel<kMaxE>, dim3(nblk), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
   }
   return cudaGetLastError();
 }
@@ -574,11 +591,11 @@ cudaError_t launch_router(const bf16* x, const bf16* Wg, int T, int h, int r, fl
 cudaError_t launch_router_small(const bf16* x, const bf16* Wg, int T, int h, int r, float beta,
                                 const KeptIds& kept, const RouteOut& out, cudaStream_t st) {
   switch (r) {
-    case 2: router_small_kernel<2><<<T, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
-    case 3: case 4: router_small_kernel<4><<<T, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
-    case 5: case 6: router_small_kernel<6><<<T, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
-    case 7: case 8: router_small_kernel<8><<<T, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
-    default: router_small_kernel<kMaxE><<<T, 256, 0, st>>>(x, Wg, T, h, r, beta, kept, out); break;
+    case 2: return launch_pdl(router_small_kernel<2>, dim3(T), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
+    case 3: case 4: return launch_pdl(router_small_kernel<4>, dim3(T), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
+    case 5: case 6: return launch_pdl(router_small_kernel<6>, dim3(T), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
+    case 7: case 8: return launch_pdl(router_small_kernel<8>, dim3(T), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
+    default: return launch_pdl(router_small_kernel<kMaxE>, dim3(T), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
   }
   return cudaGetLastError();
 }
@@ -587,26 +604,23 @@ cudaError_t launch_permute_small(const int32_t* idx, const uint8_t* skipped, int
                                  Meta* meta, int32_t* pair_pos, int32_t* row_token,
                                  int32_t* s_count, int32_t* s_nskipped, int32_t* s_ntouched,
                                  const KeptIds& kept, int E, cudaStream_t st) {
-  permute_small_kernel<<<1, kDecodeMaxT, 0, st>>>(idx, skipped, T, r, pad, meta, pair_pos, row_token,
-                                                  s_count, s_nskipped, s_ntouched, kept, E);
-  return cudaGetLastError();
+  return launch_pdl(permute_small_kernel, dim3(1), dim3(kDecodeMaxT), 0, st, idx, skipped, T, r, pad,
+                    meta, pair_pos, row_token, s_count, s_nskipped, s_ntouched, kept, E);
 }
 
 cudaError_t launch_scan(const int32_t* blk_hist, int nblk, int r, int pad, int32_t* blk_base,
                         Meta* meta, int32_t* s_count, int32_t* s_nskipped, int32_t* s_ntouched,
                         const KeptIds& kept, int E, cudaStream_t st) {
-  scan_kernel<<<1, 1024, 0, st>>>(blk_hist, nblk, r, pad, blk_base, meta, s_count, s_nskipped,
-                                  s_ntouched, kept, E);
-  return cudaGetLastError();
+  return launch_pdl(scan_kernel, dim3(1), dim3(1024), 0, st, blk_hist, nblk, r, pad, blk_base, meta,
+                    s_count, s_nskipped, s_ntouched, kept, E);
 }
 
 cudaError_t launch_scatter(const int32_t* idx, const uint8_t* skipped, const int32_t* blk_base,
                            const Meta* meta, int T, int32_t* pair_pos, int32_t* row_token,
                            cudaStream_t st) {
   const int nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
-  scatter_kernel<<<nblk, 2 * kRouteTokPerBlock, 0, st>>>(idx, skipped, blk_base, meta, T, pair_pos,
-                                                         row_token);
-  return cudaGetLastError();
+  return launch_pdl(scatter_kernel, dim3(nblk), dim3(2 * kRouteTokPerBlock), 0, st, idx, skipped,
+                    blk_base, meta, T, pair_pos, row_token);
 }
 
 cudaError_t launch_gather(const bf16* x, const int32_t* row_token, const Meta* meta, int h,
@@ -614,20 +628,20 @@ cudaError_t launch_gather(const bf16* x, const int32_t* row_token, const Meta* m
   int blocks = (cap_rows + 7) / 8;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  gather_kernel<<<blocks, 256, 0, st>>>(x, row_token, meta, h, xperm);
-  return cudaGetLastError();
+  return launch_pdl(gather_kernel, dim3(blocks), dim3(256), 0, st, x, row_token, meta, h, xperm);
 }
 
 cudaError_t launch_combine(const float* O, int ksplit, size_t split_stride, const int32_t* pair_pos,
                            const float* wn, const bf16* residual, int T, int h, bf16* y,
                            cudaStream_t st) {
-  combine_kernel<<<T, 128, 0, st>>>(O, ksplit, split_stride, pair_pos, wn, residual, T, h, y);
-  return cudaGetLastError();
+  int ychunks = ((h >> 3) + 127) / 128;
+  if (T > 4096) ychunks = 1;  // plenty of blocks already
+  return launch_pdl(combine_kernel, dim3(T, ychunks), dim3(128), 0, st, O, ksplit, split_stride,
+                    pair_pos, wn, residual, T, h, y);
 }
 
 cudaError_t launch_rmsnorm(const bf16* x, int T, int h, float eps, bf16* out, cudaStream_t st) {
-  rmsnorm_kernel<<<T, 256, 0, st>>>(x, T, h, eps, out);
-  return cudaGetLastError();
+  return launch_pdl(rmsnorm_kernel, dim3(T), dim3(256), 0, st, x, T, h, eps, out);
 }
 
 cudaError_t launch_set_dense_meta(Meta* meta, int E, int rows_per_expert, int off_stride,
