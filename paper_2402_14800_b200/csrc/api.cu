@@ -60,7 +60,7 @@ struct Workspace {
   // GEMM scratch (capacity in permuted rows)
   int cap_rows = 0;
   int map_h = 0, map_f = 0;
-  Buf row_token, xperm, act, O;
+  Buf row_token, xperm, act, O, tail;
   CUtensorMap tok_x[4], tok_act[4];  // boxes of 16/32/64/128 rows over xperm and act
   // search scratch
   Buf s_logits, s_yall, s_act, s_subsets, s_partial, s_loss_sq, s_losses, s_xpad, s_meta;
@@ -179,6 +179,7 @@ int ensure_gemm(moe_layer* L, int T) {
   if ((rc = grow(L, L->ws->xperm, (size_t)need * L->h * 2))) return rc;
   if ((rc = grow(L, L->ws->act, (size_t)need * L->f * 2))) return rc;
   if ((rc = grow(L, L->ws->O, need_O * 4))) return rc;
+  if ((rc = grow(L, L->ws->tail, kTailBufferBytes))) return rc;
   L->ws->cap_rows = need;
   L->ws->map_h = L->h;
   L->ws->map_f = L->f;
@@ -294,6 +295,7 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   gu.a_off_mul = 1; gu.out_off_mul = 1; gu.out_ld = L->f; gu.out = L->ws->act.p;
   dn.a_off_mul = 1; dn.out_off_mul = 1; dn.out_ld = L->h; dn.out = L->ws->O.p;
   const bool wm = dec && !L->debug_simt;
+  if (wm) { gu.tail = (float*)L->ws->tail.p; dn.tail = (float*)L->ws->tail.p; }
   const int ksplit = wm ? ksplit_for(L) : 1;
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;
@@ -424,7 +426,7 @@ void moe_layer_destroy(moe_layer_t* L) {
   if (!L) return;
   cudaStreamSynchronize(L->stream);
   Buf* bufs[] = {&L->own.idx, &L->own.wn, &L->own.ratio, &L->own.skipped, &L->own.blk_hist, &L->own.blk_base, &L->own.pair_pos,
-                 &L->own.meta, &L->own.status, &L->own.sel, &L->own.row_token, &L->own.xperm, &L->own.act, &L->own.O,
+                 &L->own.meta, &L->own.status, &L->own.sel, &L->own.row_token, &L->own.xperm, &L->own.act, &L->own.O, &L->own.tail,
                  &L->own.s_logits, &L->own.s_yall, &L->own.s_act, &L->own.s_subsets, &L->own.s_partial, &L->own.s_loss_sq,
                  &L->own.s_losses, &L->own.s_xpad, &L->own.s_meta, &L->own.hx, &L->own.hy, &L->own.xn};
   for (Buf* b : bufs) release(L, *b);

@@ -129,7 +129,10 @@ struct GemmArgs {
   void* out;               // bf16 activations / fp32 outputs / bf16 expert outputs
   long long split_stride;  // elements between split-K partial planes (decode down-proj)
   int* status;             // device error word
+  float* tail;             // weight-major kernel: partial tiles of K-sliced tail items, or null
 };
+
+constexpr size_t kTailBufferBytes = (size_t)256 * 128 * 128 * 4;  // one 64 KB slot per CTA
 
 int gemm_init_driver_api();  // resolves cuTensorMapEncodeTiled; 0 on success
 int make_map_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows);

@@ -441,14 +441,61 @@ constexpr int WM_BN = 128;
 
 struct ItemW {
   int c, mt, ks, tok_row, out_row, cnt, bucket, kb0, kb1;
+  int tail_slot;  // >= 0: this is one K-slice of a tail item and goes to the tail buffer
 };
 
-__device__ __forceinline__ void decode_item_w(const Meta& m, const GemmArgs& a, int item, int Mt,
-                                              int KS, int kb_per_item, int KB, ItemW& w) {
-  const int ks = item % KS;
-  const int rest = item / KS;
-  const int mt = rest % Mt;
-  const int rt = rest / Mt;
+// Work list of the weight-major kernel.  The base items (expert row tile x weight tile x
+// k-chunk) are dealt round-robin to the `grid` CTAs.  When the last round would be less than
+// half full, its `rem` items are cut into `KSt` K-slices each, so that the last round costs
+// 1/KSt of an item instead of a whole one; the slices leave fp32 partial tiles in the tail
+// buffer and tail_fixup_kernel folds them into the regular output.
+struct SchedW {
+  int Mt, KS, KB, kb_per_item;
+  int n_base, full, rem, KSt, kbs, n_total;
+};
+
+__device__ __forceinline__ SchedW make_sched_w(const Meta& m, const GemmArgs& a, int kb_per_item,
+                                               int grid) {
+  SchedW s;
+  s.KB = (a.K + BK - 1) / BK;
+  s.kb_per_item = kb_per_item;
+  s.KS = (s.KB + kb_per_item - 1) / kb_per_item;
+  s.Mt = (a.n_w_rows + 127) / 128;
+  s.n_base = m.tile_prefix[a.r] * s.Mt * s.KS;
+  s.full = (s.n_base / grid) * grid;
+  s.rem = s.n_base - s.full;
+  s.KSt = 1;
+  s.kbs = kb_per_item;
+  if (a.tail != nullptr && s.rem > 0 && 2 * s.rem <= grid) {
+    int kst = grid / s.rem;
+    const int cap = kb_per_item / 4 > 1 ? kb_per_item / 4 : 1;  // slices of at least 4 k-blocks
+    if (kst > cap) kst = cap;
+    s.kbs = (kb_per_item + kst - 1) / kst;
+    s.KSt = (kb_per_item + s.kbs - 1) / s.kbs;
+  }
+  if (s.KSt <= 1) {
+    s.KSt = 1;
+    s.full = s.n_base;
+    s.rem = 0;
+  }
+  s.n_total = s.full + s.rem * s.KSt;
+  return s;
+}
+
+__device__ __forceinline__ void decode_item_w(const Meta& m, const GemmArgs& a, const SchedW& s,
+                                              int item, ItemW& w) {
+  int base = item, sub = 0;
+  w.tail_slot = -1;
+  if (item >= s.full) {
+    const int j = item - s.full;
+    base = s.full + j / s.KSt;
+    sub = j - (j / s.KSt) * s.KSt;
+    w.tail_slot = j;
+  }
+  const int ks = base % s.KS;
+  const int rest = base / s.KS;
+  const int mt = rest % s.Mt;
+  const int rt = rest / s.Mt;
   int c = 0;
   while (c + 1 < a.r && m.tile_prefix[c + 1] <= rt) ++c;
   const int n0 = (rt - m.tile_prefix[c]) * WM_BN;
@@ -459,9 +506,15 @@ __device__ __forceinline__ void decode_item_w(const Meta& m, const GemmArgs& a, 
   w.bucket = w.cnt <= 16 ? 0 : (w.cnt <= 32 ? 1 : (w.cnt <= 64 ? 2 : 3));
   w.tok_row = a.a_row_base + a.a_off_mul * m.off[c] + n0;
   w.out_row = a.out_row_base + a.out_off_mul * m.off[c] + n0;
-  w.kb0 = ks * kb_per_item;
-  w.kb1 = min(KB, w.kb0 + kb_per_item);
+  w.kb0 = ks * s.kb_per_item;
+  w.kb1 = min(s.KB, w.kb0 + s.kb_per_item);
+  if (w.tail_slot >= 0) {
+    w.kb0 += sub * s.kbs;
+    w.kb1 = min(w.kb1, w.kb0 + s.kbs);  // may be empty for a short last k-chunk
+  }
 }
+
+constexpr int kTailSlotFloats = 128 * WM_BN;  // one partial tile: [token][weight row] fp32
 
 template <bool GATE_UP>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -488,10 +541,8 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   const uint32_t tmem_base = *(volatile uint32_t*)&bars.tmem_base;
   volatile int* abort_flag = &bars.abort_flag;
 
-  const int KB = (args.K + BK - 1) / BK;
-  const int KS = (KB + kb_per_item - 1) / kb_per_item;
-  const int Mt = (args.n_w_rows + 127) / 128;
-  const int n_items = s_meta.tile_prefix[args.r] * Mt * KS;
+  const SchedW sched = make_sched_w(s_meta, args, kb_per_item, (int)gridDim.x);
+  const int n_items = sched.n_total;
   uint32_t issued = 0;
 
   if (warp == 0) {
@@ -499,7 +550,8 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
     bool ok = true;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
       ItemW w;
-      decode_item_w(s_meta, args, item, Mt, KS, kb_per_item, KB, w);
+      decode_item_w(s_meta, args, sched, item, w);
+      if (w.kb0 >= w.kb1) continue;
       const uint32_t bytes = WM_A_BYTES + (16u << w.bucket) * 128u;
       for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
         const uint32_t s = it % WM_NS, ph = (it / WM_NS) & 1u;
@@ -519,9 +571,10 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   } else if (warp == 1) {
     uint32_t it = 0, tile_it = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile_it) {
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
       ItemW w;
-      decode_item_w(s_meta, args, item, Mt, KS, kb_per_item, KB, w);
+      decode_item_w(s_meta, args, sched, item, w);
+      if (w.kb0 >= w.kb1) continue;
       const uint32_t idesc = idesc_bf16(128, 16 << w.bucket);
       const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_empty[buf]), bph ^ 1u, abort_flag));
@@ -545,14 +598,16 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
         }
         __syncwarp();
       }
+      ++tile_it;
     }
   } else {
     const int wq = warp & 3;
     uint32_t tile_it = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile_it) {
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
       ItemW w;
-      decode_item_w(s_meta, args, item, Mt, KS, kb_per_item, KB, w);
+      decode_item_w(s_meta, args, sched, item, w);
+      if (w.kb0 >= w.kb1) continue;
       const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_full[buf]), bph, abort_flag));
       if (!ok) break;
@@ -560,7 +615,21 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
       const uint32_t taddr = tmem_base + ((uint32_t)(32 * wq) << 16) + buf * WM_BN;
       const int wrow = w.mt * 128 + 32 * wq + lane;  // weight row held by this lane
       const int nchunk = (w.cnt + 15) >> 4;
-      if (GATE_UP) {
+      if (w.tail_slot >= 0) {
+        // K-slice of a tail item: raw fp32 partial tile [token][weight row of the tile]
+        float* outp = args.tail + (size_t)w.tail_slot * kTailSlotFloats + 32 * wq + lane;
+#pragma unroll 1
+        for (int j = 0; j < nchunk; ++j) {
+          uint32_t v[16];
+          tmem_ld16(taddr + 16 * j, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int n = 16 * j + i;
+            if (n < w.cnt) outp[n * 128] = __uint_as_float(v[i]);
+          }
+        }
+      } else if (GATE_UP) {
         // lanes 0-15 hold gate rows, lanes 16-31 the up rows of the same 16 features
         const int feat = (wrow >> 5) * kInterleave + (lane & 15);
         const bool lane_ok = (lane < 16) && (w.mt * 128 + 32 * wq < args.n_w_rows);
@@ -598,9 +667,61 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[buf]));
+      ++tile_it;
     }
   }
   teardown<WM_NS, 256>(bars, tmem_base, issued, args.status);
+}
+
+// Folds the K-slices of the tail items into the regular output: the gate/up variant sums the
+// slices and applies silu(g) * u, the down variant sums them into the item's split-K plane.
+template <bool GATE_UP>
+__global__ void __launch_bounds__(128)
+tail_fixup_kernel(const GemmArgs args, int kb_per_item, int gemm_grid) {
+  __shared__ Meta s_meta;
+  pdl_launch_dependents();
+  pdl_wait();
+  for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
+    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
+  __syncthreads();
+  const SchedW sched = make_sched_w(s_meta, args, kb_per_item, gemm_grid);
+  if ((int)blockIdx.x >= sched.rem) return;
+  ItemW w;
+  // slices of this tail item, in slice order; empty slices were never written
+  int nslice = 0;
+  for (int sub = 0; sub < sched.KSt; ++sub) {
+    decode_item_w(s_meta, args, sched, sched.full + (int)blockIdx.x * sched.KSt + sub, w);
+    if (w.kb0 < w.kb1) nslice = sub + 1;
+  }
+  decode_item_w(s_meta, args, sched, sched.full + (int)blockIdx.x * sched.KSt, w);
+  const float* slot0 = args.tail + (size_t)(blockIdx.x * sched.KSt) * kTailSlotFloats;
+  if (GATE_UP) {
+    // 64 features per tile: rows 32q + s are gate, 32q + 16 + s up
+    for (int idx = threadIdx.x; idx < w.cnt * 64; idx += blockDim.x) {
+      const int n = idx >> 6, fj = idx & 63;
+      const int q = fj >> 4, sft = fj & 15;
+      if (w.mt * 128 + 32 * q >= args.n_w_rows) continue;
+      float g = 0.f, u = 0.f;
+      for (int sub = 0; sub < nslice; ++sub) {
+        const float* t = slot0 + (size_t)sub * kTailSlotFloats + n * 128;
+        g += t[32 * q + sft];
+        u += t[32 * q + 16 + sft];
+      }
+      const int feat = (w.mt * 4 + q) * kInterleave + sft;
+      reinterpret_cast<bf16*>(args.out)[(long long)(w.out_row + n) * args.out_ld + feat] =
+          __float2bfloat16_rn(silu_mul(g, u));
+    }
+  } else {
+    for (int idx = threadIdx.x; idx < w.cnt * 128; idx += blockDim.x) {
+      const int n = idx >> 7, col = idx & 127;
+      const int wrow = w.mt * 128 + col;
+      if (wrow >= args.n_w_rows) continue;
+      float v = 0.f;
+      for (int sub = 0; sub < nslice; ++sub) v += slot0[(size_t)sub * kTailSlotFloats + n * 128 + col];
+      reinterpret_cast<float*>(args.out)[(long long)w.ks * args.split_stride +
+                                         (long long)(w.out_row + n) * args.out_ld + wrow] = v;
+    }
+  }
 }
 
 // ------------------------------------------------------------ CUDA-core debug kernels
@@ -738,9 +859,16 @@ cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps&
 cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
                                   int kb_per_item, cudaStream_t st) {
   const int grid = g_num_sms > 0 ? g_num_sms : 148;
-  if (gate_up)
-    return launch_pdl(gemm_weights_m_kernel<true>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a, kb_per_item);
-  return launch_pdl(gemm_weights_m_kernel<false>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a, kb_per_item);
+  if (gate_up) {
+    cudaError_t e = launch_pdl(gemm_weights_m_kernel<true>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
+                               kb_per_item);
+    if (e != cudaSuccess || !a.tail) return e;
+    return launch_pdl(tail_fixup_kernel<true>, dim3(grid / 2), dim3(128), 0, st, a, kb_per_item, grid);
+  }
+  cudaError_t e = launch_pdl(gemm_weights_m_kernel<false>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
+                             kb_per_item);
+  if (e != cudaSuccess || !a.tail) return e;
+  return launch_pdl(tail_fixup_kernel<false>, dim3(grid / 2), dim3(128), 0, st, a, kb_per_item, grid);
 }
 
 cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,
