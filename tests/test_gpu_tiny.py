@@ -218,3 +218,45 @@ def test_rmsnorm_and_stack(setup):
     assert np.quantile(err, 0.97) <= P.Y_REL_L2_TOL
     for l in layers:
         l.close()
+
+
+@pytest.mark.parametrize("h,f,E,kept,T", [
+    (192, 320, 4, 0b1111, 300),     # ragged K and N tiles, few experts
+    (192, 320, 4, 0b1011, 40),
+    (64, 64, 16, 0xFFFF, 513),      # smallest shapes, 16 experts
+    (256, 192, 16, 0xF0F3, 200),    # 10 of 16 experts kept (generic router path)
+    (128, 448, 2, 0b11, 129),       # every token uses both experts
+])
+def test_forward_other_shapes(h, f, E, kept, T):
+    build.build()
+    W = synth.make_layer_weights(h, f, E, seed=31)
+    b = synth.bf16_bits
+    host = dict(Wg=b(W.W_gate), W1=b(W.W1), W3=b(W.W3), W2=b(W.W2))
+    x = synth.make_tokens(T, h, seed=32)
+    beta = 0.35
+    ora = O.moe_forward(b(x), host["Wg"], host["W1"], host["W3"], host["W2"], kept, beta)
+    ora["logits"] = O.route(b(x), host["Wg"], kept, beta)["logits"]
+    layer = binding.MoeLayer(W.W_gate.to(DEV), W.W1.to(DEV), W.W3.to(DEV), W.W2.to(DEV), kept)
+    stats = binding.RoutingStats(T, E, DEV)
+    y = layer.forward(x.to(DEV), beta, stats=stats)
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+    gi, gs = stats.idx.cpu().numpy(), stats.skipped.cpu().numpy()
+    P.check_routing(gi, gs, stats.wn.cpu().numpy(), stats.ratio.cpu().numpy(), ora, kept, beta)
+    ok = (gi == ora["idx"]).all(1) & (gs == ora["skipped"])
+    P.check_outputs(b(y), ora["y"], ok)
+    layer.close()
+
+
+@pytest.mark.parametrize("E,r", [(4, 2), (4, 3), (16, 14), (16, 15), (6, 3)])
+def test_prune_search_other_expert_counts(E, r):
+    build.build()
+    h, f, T = 128, 192, 150
+    W = synth.make_layer_weights(h, f, E, seed=41)
+    b = synth.bf16_bits
+    x = synth.make_tokens(T, h, seed=42)
+    ora = O.prune_search_allexperts(b(x), b(W.W_gate), b(W.W1), b(W.W3), b(W.W2), r)
+    layer = binding.MoeLayer(W.W_gate.to(DEV), W.W1.to(DEV), W.W3.to(DEV), W.W2.to(DEV))
+    losses, best = layer.prune_search(x.to(DEV), r)
+    layer.close()
+    P.check_search(losses, best, ora)
