@@ -411,6 +411,22 @@ def run_ours(a):
         cpu = {"value": n_sample * per_unit / dt, "unit": metric_unit(a)[1], "cores": O.num_threads(),
                "kind": "oracle", "sample": "%d of %d tokens, one pass, %.1f s" % (n_sample, T, dt)}
 
+    # reconstruction loss of the searched subset against the pruning baselines of the paper's
+    # comparison (activation frequency, random), all on the same synthetic calibration batch
+    baselines = None
+    if a.workload == "search" and rank == 0:
+        from itertools import combinations
+        counts = layer.coselection(x)
+        baselines = {}
+        for r_ in (6, 4):
+            losses, best = layer.prune_search(x, r_)
+            masks = [sum(1 << i for i in c) for c in combinations(range(E), r_)]
+            fmask = layer.frequency_subset(counts, r_)
+            baselines["r%d" % r_] = {"searched_subset": best, "searched_loss": min(losses),
+                                     "frequency_subset": fmask, "frequency_loss": losses[masks.index(fmask)],
+                                     "random_mean_loss": float(np.mean(losses)),
+                                     "worst_loss": max(losses)}
+
     if rank == 0:
         metric, unit = metric_unit(a)
         gpu_launches = launches_per_step * a.steps if launches_per_step else None
@@ -430,6 +446,8 @@ def run_ours(a):
             "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "roofline": roofline,
             "cpu_baseline": cpu, "stages": stages,
         }
+        if baselines:
+            line["pruning_baselines"] = baselines
         print(json.dumps(line), flush=True)
     layer.close()
     if world > 1:

@@ -168,6 +168,23 @@ int moe_prune_search(moe_layer_t* layer, const void* x_calib, int T, int r, floa
 int moe_calibrate_beta_noalloc(const void* W_gate_kept, const void* x, int T, int h, int r,
                                void* cuda_stream, float* beta_out);
 
+/*
+ * Expert co-selection counts (App. A.1): counts[a][b] (host, E x E int32, row a) is
+ * the number of the T tokens whose largest routing weight is expert a and second
+ * largest expert b under this layer's router, original expert ids, no skipping.
+ * The activation frequency of expert e is the sum of row e and column e.
+ * x [T][h] bf16 device.  Synchronises the handle's stream.
+ */
+int moe_coselection(moe_layer_t* layer, const void* x, int T, int32_t* counts);
+
+/*
+ * The activation-frequency pruning baseline (Sec. 4.1, "Comparison with Other
+ * Expert Pruning Baselines"): bitmask of the r experts with the highest
+ * activation frequency in `counts` (as written by moe_coselection; ties to the
+ * lower index).  Host only.  Returns 0 for invalid arguments.
+ */
+uint32_t moe_frequency_subset(const int32_t* counts, int E, int r);
+
 /* Number of subsets moe_prune_search scores: C(E, r), 0 if out of range. */
 long moe_num_subsets(int E, int r);
 

@@ -215,6 +215,43 @@ int oracle_all_experts(const uint16_t *x, const uint16_t *W1, const uint16_t *W3
   return 0;
 }
 
+/* Expert co-selection counts (App. A.1): counts[a][b] = number of tokens whose largest
+ * routing weight is expert a and second largest expert b (all experts kept, no skipping).
+ * The activation frequency of expert e, which the frequency-based pruning baseline of
+ * Sec. 4.1 ranks by, is the sum of row e and column e. */
+int oracle_coselection(const uint16_t *x, const uint16_t *Wg, int T, int h, int E, int64_t *counts) {
+  if (E < 2 || E > ORACLE_MAX_E) return -1;
+  for (int i = 0; i < E * E; ++i) counts[i] = 0;
+  uint32_t full = (1u << E) - 1u;
+  for (int t = 0; t < T; ++t) {
+    float l[ORACLE_MAX_E], wr[2], wnn[2], rt;
+    int32_t id[2];
+    uint8_t sk;
+    router_logits(x + (size_t)t * h, Wg, h, E, l);
+    route_token(l, E, full, 0.0f, id, wr, wnn, &rt, &sk);
+    counts[id[0] * E + id[1]] += 1;
+  }
+  return 0;
+}
+
+/* Frequency baseline: keep the r experts with the highest activation frequency
+ * (ties to the lower index). */
+uint32_t oracle_frequency_subset(const int64_t *counts, int E, int r) {
+  int64_t freq[ORACLE_MAX_E];
+  for (int e = 0; e < E; ++e) {
+    freq[e] = 0;
+    for (int b = 0; b < E; ++b) freq[e] += counts[e * E + b] + counts[b * E + e];
+  }
+  uint32_t mask = 0;
+  for (int k = 0; k < r; ++k) {
+    int best = -1;
+    for (int e = 0; e < E; ++e)
+      if (!((mask >> e) & 1u) && (best < 0 || freq[e] > freq[best])) best = e;
+    mask |= 1u << best;
+  }
+  return mask;
+}
+
 /* --------------------------------------------------------------- forward */
 
 /* Pruned + skipping MoE layer forward (Eq. 2 with the routing above):

@@ -155,6 +155,26 @@ def moe_forward(x, Wg, W1, W3, W2, kept_mask: int, beta: float, residual=None):
     return out
 
 
+def coselection(x, Wg) -> np.ndarray:
+    """counts[E,E] int64: tokens with top-1 expert a and top-2 expert b."""
+    x = _u16(x)
+    T, h = x.shape
+    Wg = _u16(Wg)
+    E = Wg.shape[0]
+    counts = np.zeros((E, E), np.int64)
+    if lib().oracle_coselection(_p(x, _u16p), _p(Wg, _u16p), T, h, E, _p(counts, _i64p)):
+        raise ValueError("oracle_coselection: invalid arguments")
+    return counts
+
+
+def frequency_subset(counts, r: int) -> int:
+    counts = np.ascontiguousarray(counts, dtype=np.int64)
+    E = counts.shape[0]
+    fn = lib().oracle_frequency_subset
+    fn.restype = ctypes.c_uint32
+    return int(fn(_p(counts, _i64p), E, r))
+
+
 def beta_median(ratio) -> float:
     ratio = np.ascontiguousarray(ratio, dtype=np.float32)
     b = ctypes.c_float(0)

@@ -64,6 +64,9 @@ def load_library(path: str | None = None):
     lib.moe_num_subsets.argtypes = [ci, ci]
     lib.moe_rmsnorm.argtypes = [vp, ci, ci, cf, vp, vp]
     lib.moe_stack_forward.argtypes = [ctypes.POINTER(vp), ci, vp, ci, ctypes.POINTER(cf), cf, vp]
+    lib.moe_coselection.argtypes = [vp, vp, ci, ctypes.POINTER(ctypes.c_int32)]
+    lib.moe_frequency_subset.restype = u32
+    lib.moe_frequency_subset.argtypes = [ctypes.POINTER(ctypes.c_int32), ci, ci]
     lib.moe_device_status.argtypes = [vp]
     lib.moe_layer_share_scratch.argtypes = [vp, vp]
     lib.moe_profile_enable.argtypes = [vp, ci]
@@ -204,6 +207,20 @@ class MoeLayer:
         best = ctypes.c_uint32(0)
         _check(load_library().moe_prune_search(self._h, x_calib.data_ptr(), T, r, losses, ctypes.byref(best)))
         return list(losses)[:n], int(best.value)
+
+    def coselection(self, x):
+        """``moe_coselection``: E x E list of lists, counts[a][b] = tokens with top-2 (a, b)."""
+        T = x.shape[0]
+        _dev_bf16(x, (T, self.h))
+        buf = (ctypes.c_int32 * (self.E * self.E))()
+        _check(load_library().moe_coselection(self._h, x.data_ptr(), T, buf))
+        return [[int(buf[a * self.E + b]) for b in range(self.E)] for a in range(self.E)]
+
+    def frequency_subset(self, counts, r: int) -> int:
+        """``moe_frequency_subset``: the activation-frequency baseline's kept mask."""
+        flat = [int(v) for row in counts for v in row]
+        buf = (ctypes.c_int32 * len(flat))(*flat)
+        return int(load_library().moe_frequency_subset(buf, self.E, r))
 
     def profile_enable(self, on: bool = True):
         _check(load_library().moe_profile_enable(self._h, int(bool(on))))

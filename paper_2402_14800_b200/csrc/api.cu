@@ -65,7 +65,7 @@ struct Workspace {
   // search scratch
   Buf s_logits, s_yall, s_act, s_subsets, s_partial, s_loss_sq, s_losses, s_xpad, s_meta;
   // host staging and stack scratch
-  Buf hx, hy, xn;
+  Buf hx, hy, xn, cosel;
 };
 
 int moe::set_error(int code, const char* fmt, ...) {
@@ -428,7 +428,7 @@ void moe_layer_destroy(moe_layer_t* L) {
   Buf* bufs[] = {&L->own.idx, &L->own.wn, &L->own.ratio, &L->own.skipped, &L->own.blk_hist, &L->own.blk_base, &L->own.pair_pos,
                  &L->own.meta, &L->own.status, &L->own.sel, &L->own.row_token, &L->own.xperm, &L->own.act, &L->own.O, &L->own.tail,
                  &L->own.s_logits, &L->own.s_yall, &L->own.s_act, &L->own.s_subsets, &L->own.s_partial, &L->own.s_loss_sq,
-                 &L->own.s_losses, &L->own.s_xpad, &L->own.s_meta, &L->own.hx, &L->own.hy, &L->own.xn};
+                 &L->own.s_losses, &L->own.s_xpad, &L->own.s_meta, &L->own.hx, &L->own.hy, &L->own.xn, &L->own.cosel};
   for (Buf* b : bufs) release(L, *b);
   for (cudaEvent_t e : L->prof_ev) cudaEventDestroy(e);
   if (L->Wg) cudaFree(L->Wg);
@@ -488,6 +488,46 @@ int moe_calibrate_beta(moe_layer_t* L, const void* x, int T, float* beta_out) {
   CUDA_TRY(cudaStreamSynchronize(L->stream));
   *beta_out = (T & 1) ? v[0] : (float)(((double)v[0] + (double)v[1]) * 0.5);
   return MOE_OK;
+}
+
+int moe_coselection(moe_layer_t* L, const void* x, int T, int32_t* counts) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  if (!x || !counts) return fail(MOE_ERR_INVALID_ARG, "x or counts is NULL");
+  if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
+  if (!aligned16(x)) return fail(MOE_ERR_INVALID_ARG, "x must be 16-byte aligned");
+  const int E = L->E;
+  memset(counts, 0, sizeof(int32_t) * E * E);
+  if (T == 0) return MOE_OK;
+  int rc;
+  if ((rc = ensure_route(L, T))) return rc;
+  if ((rc = grow(L, L->ws->cosel, (size_t)E * E * 4))) return rc;
+  RouteOut ro;
+  memset(&ro, 0, sizeof(ro));
+  ro.idx = (int32_t*)L->ws->idx.p; ro.wn = (float*)L->ws->wn.p; ro.ratio = (float*)L->ws->ratio.p;
+  ro.skipped = (uint8_t*)L->ws->skipped.p;
+  CUDA_TRY(cudaMemsetAsync(L->ws->cosel.p, 0, (size_t)E * E * 4, L->stream));
+  CUDA_TRY(launch_router((const bf16*)x, L->Wg, T, L->h, L->r, 0.f, L->kept, ro, L->stream));
+  CUDA_TRY(launch_coselection(ro.idx, T, E, L->kept, (int32_t*)L->ws->cosel.p, L->stream));
+  CUDA_TRY(cudaMemcpyAsync(counts, L->ws->cosel.p, (size_t)E * E * 4, cudaMemcpyDeviceToHost, L->stream));
+  CUDA_TRY(cudaStreamSynchronize(L->stream));
+  return MOE_OK;
+}
+
+uint32_t moe_frequency_subset(const int32_t* counts, int E, int r) {
+  if (!counts || E < 2 || E > kMaxE || r < 1 || r > E) return 0;
+  long long freq[kMaxE];
+  for (int e = 0; e < E; ++e) {
+    freq[e] = 0;
+    for (int b = 0; b < E; ++b) freq[e] += (long long)counts[e * E + b] + counts[b * E + e];
+  }
+  uint32_t mask = 0;
+  for (int k = 0; k < r; ++k) {
+    int best = -1;
+    for (int e = 0; e < E; ++e)
+      if (!((mask >> e) & 1u) && (best < 0 || freq[e] > freq[best])) best = e;
+    mask |= 1u << best;
+  }
+  return mask;
 }
 
 int moe_prune_search(moe_layer_t* L, const void* x_calib, int T, int r, float* losses,

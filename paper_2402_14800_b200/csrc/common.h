@@ -103,6 +103,8 @@ cudaError_t launch_gather(const bf16* x, const int32_t* row_token, const Meta* m
 cudaError_t launch_combine(const float* O, int ksplit, size_t split_stride, const int32_t* pair_pos,
                            const float* wn, const bf16* residual, int T, int h, bf16* y,
                            cudaStream_t st);
+cudaError_t launch_coselection(const int32_t* idx, int T, int E, const KeptIds& kept, int32_t* counts,
+                               cudaStream_t st);
 cudaError_t launch_rmsnorm(const bf16* x, int T, int h, float eps, bf16* out, cudaStream_t st);
 cudaError_t launch_set_dense_meta(Meta* meta, int E, int rows_per_expert, int off_stride,
                                   cudaStream_t st);

@@ -446,6 +446,25 @@ combine_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
   }
 }
 
+// --------------------------------------------------------------------------- co-selection
+
+// counts[a][b] += 1 for every token whose top-2 is (a, b) (App. A.1).  Integer counts: block
+// histograms in shared memory, then integer atomics, so the result is exact and order-free.
+__global__ void __launch_bounds__(256)
+coselection_kernel(const int32_t* __restrict__ idx, int T, int E, KeptIds kept,
+                   int32_t* __restrict__ counts) {
+  __shared__ int s_c[kMaxE * kMaxE];
+  for (int i = threadIdx.x; i < kMaxE * kMaxE; i += blockDim.x) s_c[i] = 0;
+  __syncthreads();
+  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < T; t += gridDim.x * blockDim.x)
+    atomicAdd(&s_c[kept.id[idx[2 * t]] * kMaxE + kept.id[idx[2 * t + 1]]], 1);
+  __syncthreads();
+  for (int i = threadIdx.x; i < kMaxE * kMaxE; i += blockDim.x) {
+    const int a = i / kMaxE, b = i % kMaxE;
+    if (a < E && b < E && s_c[i]) atomicAdd(&counts[a * E + b], s_c[i]);
+  }
+}
+
 // ------------------------------------------------------------------------------- rmsnorm
 
 __global__ void __launch_bounds__(256)
@@ -638,6 +657,14 @@ cudaError_t launch_combine(const float* O, int ksplit, size_t split_stride, cons
   if (T > 4096) ychunks = 1;  // plenty of blocks already
   return launch_pdl(combine_kernel, dim3(T, ychunks), dim3(128), 0, st, O, ksplit, split_stride,
                     pair_pos, wn, residual, T, h, y);
+}
+
+cudaError_t launch_coselection(const int32_t* idx, int T, int E, const KeptIds& kept, int32_t* counts,
+                               cudaStream_t st) {
+  int blocks = (T + 255) / 256;
+  if (blocks > 148 * 4) blocks = 148 * 4;
+  coselection_kernel<<<blocks, 256, 0, st>>>(idx, T, E, kept, counts);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_rmsnorm(const bf16* x, int T, int h, float eps, bf16* out, cudaStream_t st) {

@@ -14,8 +14,8 @@ namespace moe {
 
 namespace {
 
-constexpr int kTokPerWarp = 8;
-constexpr int kMaxBlocks = 148 * 8;
+constexpr int kTokPerWarp = 2;
+constexpr int kMaxBlocks = 148 * 16;
 
 __device__ __forceinline__ void unpack8f(const uint4& v, float* f) {
   f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);

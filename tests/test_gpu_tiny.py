@@ -260,3 +260,26 @@ def test_prune_search_other_expert_counts(E, r):
     losses, best = layer.prune_search(x.to(DEV), r)
     layer.close()
     P.check_search(losses, best, ora)
+
+
+def test_coselection_and_frequency_baseline(setup):
+    host, dev = setup
+    T = 1500
+    x = synth.make_tokens(T, H, seed=12)
+    want = O.coselection(synth.bf16_bits(x), host["Wg"])
+    ties = int(P.near_tie_tokens(O.route(synth.bf16_bits(x), host["Wg"], FULL, 0.0)["logits"], FULL).sum())
+    layer = make_layer(dev)
+    got = np.array(layer.coselection(x.to(DEV)), np.int64)
+    assert got.sum() == T and np.trace(got) == 0
+    assert np.abs(got - want).sum() <= 2 * ties
+    for r in (6, 4):
+        assert layer.frequency_subset(want.tolist(), r) == O.frequency_subset(want, r)
+    # the searched subset is never worse than the frequency baseline's or a random subset
+    losses, best = layer.prune_search(x.to(DEV), 6)
+    subsets = O.enumerate_subsets(E, 6).tolist()
+    freq_loss = losses[subsets.index(O.frequency_subset(want, 6))]
+    assert min(losses) <= freq_loss and min(losses) <= float(np.mean(losses))
+    pruned = make_layer(dev, 0b00111111)
+    assert np.array(pruned.coselection(x.to(DEV)))[6:, :].sum() == 0
+    pruned.close()
+    layer.close()

@@ -319,3 +319,26 @@ def test_rmsnorm_matches_numpy(cfg0):
     x = D.bits_to_f64(cfg0["x"])
     want = D.to_bf16_bits(x / np.sqrt((x * x).mean(1, keepdims=True) + 1e-5))
     assert np.array_equal(O.rmsnorm(cfg0["x"], 1e-5), want)
+
+
+# ------------------------------------------------------------------- baselines
+
+def test_coselection_counts_and_frequency_subset(cfg0, dense):
+    """App. A.1 co-selection map and the activation-frequency baseline of Sec. 4.1."""
+    counts = O.coselection(cfg0["x"], cfg0["Wg"])
+    assert counts.sum() == T and np.trace(counts) == 0
+    e0, e1, gap01, gap12 = D.top2(dense["l"], FULL)
+    want = np.zeros((E, E), np.int64)
+    np.add.at(want, (e0, e1), 1)
+    n_tie = int(((gap01 <= 1e-3) | (gap12 <= 1e-3)).sum())
+    assert np.abs(counts - want).sum() <= 2 * n_tie
+    freq = counts.sum(0) + counts.sum(1)
+    assert freq.sum() == 2 * T
+    for r in (6, 4, 2):
+        mask = O.frequency_subset(counts, r)
+        order = sorted(range(E), key=lambda e: (-freq[e], e))[:r]
+        assert mask == sum(1 << e for e in order)
+    # a tie in frequency keeps the lower index
+    c = np.zeros((4, 4), np.int64)
+    c[0, 1] = c[2, 3] = 5
+    assert O.frequency_subset(c, 2) == 0b0011
