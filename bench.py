@@ -478,9 +478,11 @@ def run_stack(a):
     x = synth.make_tokens(T, H, seed=1, device=dev)
     state = synth.make_tokens(a.cal_tokens, H, seed=1001, device=dev)
     layers, betas, masks, search_ms = [], [], [], 0.0
+    state_p = state.clone() if (r < 8 and a.search_mode == "progressive") else None
     for l in range(NL):
         W = synth.make_layer_weights(H, F, E, seed=100 + l, device=dev)
         xn = binding.rmsnorm(state)
+        xn_cal = xn
         if r == 8:
             layer = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, 0xFF)
             if layers:
@@ -491,7 +493,15 @@ def run_stack(a):
             full = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, 0xFF)
             torch.cuda.synchronize(dev)
             t0 = time.perf_counter()
-            _, mask = full.prune_search(xn, r)
+            if state_p is None:
+                # layer-wise: every layer is searched on the unpruned stack's states
+                _, mask = full.prune_search(xn, r)
+            else:
+                # progressive: input from the pruned stack so far, target from the unpruned stack
+                F_ref = full.forward(xn, 0.0).float()
+                xn_cal = binding.rmsnorm(state_p)
+                _, mask = full.prune_search_progressive(xn_cal, F_ref, r)
+                del F_ref
             search_ms += 1e3 * (time.perf_counter() - t0)
             state = full.forward(xn, 0.0, residual=state)
             torch.cuda.synchronize(dev)
@@ -499,10 +509,22 @@ def run_stack(a):
             layer = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, mask)
             if layers:
                 layer.share_scratch(layers[0])
-        betas.append(layer.calibrate_beta(xn) if a.beta == "calibrated" else 0.0)
+            if state_p is not None:
+                state_p = layer.forward(xn_cal, 0.0, residual=state_p)
+        betas.append(layer.calibrate_beta(xn_cal) if a.beta == "calibrated" else 0.0)
         masks.append(mask)
         layers.append(layer)
         del W
+    # how far the pruned stack's calibration states ended up from the unpruned stack's
+    drift = None
+    if state_p is not None:
+        drift = float((state_p.float() - state.float()).norm() / state.float().norm())
+    elif r < 8:
+        sp = synth.make_tokens(a.cal_tokens, H, seed=1001, device=dev)
+        for layer in layers:
+            sp = layer.forward(binding.rmsnorm(sp), 0.0, residual=sp)
+        drift = float((sp.float() - state.float()).norm() / state.float().norm())
+        del sp
     del state, xn
     stream = torch.cuda.Stream(dev)
     for layer in layers:
@@ -594,6 +616,8 @@ def run_stack(a):
                        "betas": [round(b, 4) for b in betas], "weight_bytes": weight_bytes,
                        "experts_touched_sum": sum(touched), "pairs_sum": sum(pairs),
                        "search_ms_total": search_ms, "calibration_tokens": a.cal_tokens,
+                       "search_mode": a.search_mode if r < 8 else None,
+                       "final_state_rel_error_vs_unpruned": drift,
                        "parallelism": "replicas x%d, no collective" % world,
                        "l2": "each layer streams its own weights (GBs), far above the 126 MB L2"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": per_layer * NL * a.steps,
@@ -617,6 +641,7 @@ def main():
     ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "search", "stack"])
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--cal-tokens", type=int, default=4096)
+    ap.add_argument("--search-mode", default="layerwise", choices=["layerwise", "progressive"])
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--beta", default="0", choices=["0", "calibrated"])
     ap.add_argument("--kept", default="full", choices=list(KEPT))

@@ -169,6 +169,18 @@ int moe_calibrate_beta_noalloc(const void* W_gate_kept, const void* x, int T, in
                                void* cuda_stream, float* beta_out);
 
 /*
+ * Progressive variant of the search (the paper's ablation of layer-wise vs
+ * progressive pruning, Sec. 4.4 "Ablation"): the pruned layer is evaluated on
+ * x_pruned, calibration states that already went through the pruned earlier
+ * layers, while the target stays the unpruned model's cached output of this
+ * layer:   losses[i] = || F'(x_pruned, C_i) - F_ref ||_F.
+ * x_pruned [T][h] bf16 device; F_ref [T][h] fp32 device (the cached layer
+ * output, without the residual); everything else as moe_prune_search.
+ */
+int moe_prune_search_progressive(moe_layer_t* layer, const void* x_pruned, const float* F_ref,
+                                 int T, int r, float* losses, uint32_t* best_subset);
+
+/*
  * Expert co-selection counts (App. A.1): counts[a][b] (host, E x E int32, row a) is
  * the number of the T tokens whose largest routing weight is expert a and second
  * largest expert b under this layer's router, original expert ids, no skipping.

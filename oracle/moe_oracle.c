@@ -497,6 +497,60 @@ int oracle_prune_search_allexperts(const uint16_t *x, const uint16_t *Wg, const 
   return 0;
 }
 
+/* Progressive variant of the search (the "progressive" row of the paper's ablation on
+ * layer-wise vs progressive pruning): the pruned layer is evaluated on x_p, the calibration
+ * states that already went through the pruned earlier layers, while the target stays the
+ * unpruned model's cached output F_ref[T][h] of this layer:
+ *   loss(C) = || F'(x_p, C) - F_ref ||_F.
+ * Expert outputs carry R3 as in the layer-wise search. */
+int oracle_prune_search_progressive(const uint16_t *x_p, const uint16_t *Wg, const uint16_t *W1,
+                                    const uint16_t *W3, const uint16_t *W2, const float *F_ref,
+                                    int T, int h, int f, int E, int r, double *losses,
+                                    double *loss_sq, uint32_t *best_subset) {
+  if (E < 2 || E > ORACLE_MAX_E || r < 2 || r > E) return -1;
+  long nC = binom(E, r);
+  uint32_t *masks = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)nC);
+  oracle_enumerate_subsets(E, r, masks);
+  uint32_t full = (1u << E) - 1u;
+  double *Yall = (double *)malloc(sizeof(double) * (size_t)T * E * h);
+  if (!Yall) { free(masks); return -2; }
+  oracle_all_experts(x_p, W1, W3, W2, T, h, f, E, full, 1, Yall);
+  double *err = (double *)malloc(sizeof(double) * (size_t)T * nC);
+#pragma omp parallel for schedule(static)
+  for (int t = 0; t < T; ++t) {
+    float l[ORACLE_MAX_E];
+    router_logits(x_p + (size_t)t * h, Wg, h, E, l);
+    int32_t idc[2];
+    float wr[2], wnC[2], rt;
+    uint8_t sk;
+    const double *Y = Yall + (size_t)t * E * h;
+    for (long c = 0; c < nC; ++c) {
+      route_token(l, E, masks[c], 0.0f, idc, wr, wnC, &rt, &sk);
+      double e2 = 0.0;
+      for (int i = 0; i < h; ++i) {
+        double Fp = (double)wnC[0] * Y[(size_t)idc[0] * h + i] + (double)wnC[1] * Y[(size_t)idc[1] * h + i];
+        double d = Fp - (double)F_ref[(size_t)t * h + i];
+        e2 += d * d;
+      }
+      err[(size_t)t * nC + c] = e2;
+    }
+  }
+  long best = 0;
+  for (long c = 0; c < nC; ++c) {
+    double sq = 0.0;
+    for (int t = 0; t < T; ++t) sq += err[(size_t)t * nC + c];
+    losses[c] = sqrt(sq);
+    if (loss_sq) loss_sq[c] = sq;
+  }
+  for (long c = 0; c < nC; ++c)
+    if (losses[c] < losses[best]) best = c;
+  if (best_subset) *best_subset = masks[best];
+  free(masks);
+  free(Yall);
+  free(err);
+  return 0;
+}
+
 /* ------------------------------------------------------------ stack glue */
 
 /* RMSNorm with unit gain: out = bf16( x / sqrt(mean(x^2) + eps) ), as placed

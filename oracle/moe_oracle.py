@@ -216,6 +216,30 @@ def prune_search_allexperts(x, Wg, W1, W3, W2, r: int):
     return _search(lib().oracle_prune_search_allexperts, x, Wg, W1, W3, W2, r)
 
 
+def prune_search_progressive(x_p, Wg, W1, W3, W2, F_ref, r: int):
+    """Progressive search: the pruned layer runs on x_p, the target is the cached F_ref[T,h] f32."""
+    x_p = _u16(x_p)
+    T, h = x_p.shape
+    Wg = _u16(Wg)
+    E = Wg.shape[0]
+    W1 = _u16(W1)
+    f = W1.shape[1]
+    W3 = _u16(W3, (E, f, h))
+    W2 = _u16(W2, (E, h, f))
+    F_ref = np.ascontiguousarray(F_ref, dtype=np.float32)
+    assert F_ref.shape == (T, h)
+    nC = comb(E, r)
+    losses = np.zeros(nC, np.float64)
+    loss_sq = np.zeros(nC, np.float64)
+    best = ctypes.c_uint32(0)
+    rc = lib().oracle_prune_search_progressive(
+        _p(x_p, _u16p), _p(Wg, _u16p), _p(W1, _u16p), _p(W3, _u16p), _p(W2, _u16p), _p(F_ref, _f32p),
+        T, h, f, E, r, _p(losses, _f64p), _p(loss_sq, _f64p), ctypes.byref(best))
+    if rc:
+        raise ValueError("oracle progressive search: invalid arguments")
+    return dict(losses=losses, loss_sq=loss_sq, best_subset=int(best.value), subsets=enumerate_subsets(E, r))
+
+
 def rmsnorm(x, eps: float = 1e-5) -> np.ndarray:
     x = _u16(x)
     T, h = x.shape

@@ -60,6 +60,7 @@ def load_library(path: str | None = None):
     lib.moe_routing_stats_bytes.argtypes = [ci, ci]
     lib.moe_calibrate_beta.argtypes = [vp, vp, ci, ctypes.POINTER(cf)]
     lib.moe_prune_search.argtypes = [vp, vp, ci, ci, ctypes.POINTER(cf), ctypes.POINTER(u32)]
+    lib.moe_prune_search_progressive.argtypes = [vp, vp, vp, ci, ci, ctypes.POINTER(cf), ctypes.POINTER(u32)]
     lib.moe_num_subsets.restype = ctypes.c_long
     lib.moe_num_subsets.argtypes = [ci, ci]
     lib.moe_rmsnorm.argtypes = [vp, ci, ci, cf, vp, vp]
@@ -231,6 +232,20 @@ class MoeLayer:
         n = ctypes.c_int(0)
         _check(load_library().moe_profile_read(self._h, ms, ctypes.byref(n)))
         return [float(v) for v in ms], int(n.value)
+
+    def prune_search_progressive(self, x_pruned, F_ref, r: int):
+        """``moe_prune_search_progressive``: F_ref is a contiguous fp32 CUDA tensor [T, h]."""
+        T = x_pruned.shape[0]
+        _dev_bf16(x_pruned, (T, self.h))
+        if not (F_ref.is_cuda and F_ref.dtype == torch.float32 and F_ref.is_contiguous()
+                and tuple(F_ref.shape) == (T, self.h)):
+            raise MoeError(-1, "F_ref must be a contiguous fp32 CUDA tensor of shape [T, h]")
+        n = comb(self.E, r) if 0 <= r <= self.E else 1
+        losses = (ctypes.c_float * max(n, 1))()
+        best = ctypes.c_uint32(0)
+        _check(load_library().moe_prune_search_progressive(self._h, x_pruned.data_ptr(), F_ref.data_ptr(),
+                                                           T, r, losses, ctypes.byref(best)))
+        return list(losses)[:n], int(best.value)
 
     def device_status(self) -> int:
         return int(load_library().moe_device_status(self._h))

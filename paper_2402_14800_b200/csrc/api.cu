@@ -530,8 +530,8 @@ uint32_t moe_frequency_subset(const int32_t* counts, int E, int r) {
   return mask;
 }
 
-int moe_prune_search(moe_layer_t* L, const void* x_calib, int T, int r, float* losses,
-                     uint32_t* best_subset) {
+static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, int T, int r,
+                       float* losses, uint32_t* best_subset) {
   if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
   if (!x_calib || !losses || !best_subset)
     return fail(MOE_ERR_INVALID_ARG, "x_calib, losses or best_subset is NULL");
@@ -620,7 +620,7 @@ int moe_prune_search(moe_layer_t* L, const void* x_calib, int T, int r, float* l
   L->prof = prof_saved;
   CUDA_TRY(launch_enumerate((const float*)L->ws->s_logits.p, (const bf16*)L->ws->s_yall.p, T, E, r, h,
                             (const uint32_t*)L->ws->s_subsets.p, (int)nC, (float*)L->ws->s_partial.p,
-                            (double*)L->ws->s_loss_sq.p, (float*)L->ws->s_losses.p, st));
+                            (double*)L->ws->s_loss_sq.p, (float*)L->ws->s_losses.p, F_ref, st));
   CUDA_TRY(cudaMemcpyAsync(losses, L->ws->s_losses.p, (size_t)nC * 4, cudaMemcpyDeviceToHost, st));
   if ((rc = check_status(L))) return rc;
   long best = 0;
@@ -628,6 +628,18 @@ int moe_prune_search(moe_layer_t* L, const void* x_calib, int T, int r, float* l
     if (losses[c] < losses[best]) best = c;
   *best_subset = masks[best];
   return MOE_OK;
+}
+
+int moe_prune_search(moe_layer_t* L, const void* x_calib, int T, int r, float* losses,
+                     uint32_t* best_subset) {
+  return search_impl(L, x_calib, nullptr, T, r, losses, best_subset);
+}
+
+int moe_prune_search_progressive(moe_layer_t* L, const void* x_pruned, const float* F_ref, int T,
+                                 int r, float* losses, uint32_t* best_subset) {
+  if (!F_ref) return fail(MOE_ERR_INVALID_ARG, "F_ref is NULL");
+  if (!aligned16(F_ref)) return fail(MOE_ERR_INVALID_ARG, "F_ref must be 16-byte aligned");
+  return search_impl(L, x_pruned, F_ref, T, r, losses, best_subset);
 }
 
 int moe_rmsnorm(const void* x, int T, int h, float eps, void* out, void* cuda_stream) {

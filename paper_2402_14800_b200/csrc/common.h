@@ -164,6 +164,6 @@ cudaError_t gemm_set_attributes();
 int enumerate_num_blocks(int T, int nC);
 cudaError_t launch_enumerate(const float* logits, const bf16* Yall, int T, int E, int r, int h,
                              const uint32_t* subsets, int nC, float* partial, double* loss_sq,
-                             float* losses, cudaStream_t st);
+                             float* losses, const float* Fref, cudaStream_t st);
 
 }  // namespace moe

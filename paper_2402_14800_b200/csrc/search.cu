@@ -34,10 +34,13 @@ __device__ __forceinline__ void pair_weights(float l_first, float l_second, floa
 }
 
 // Squared errors of all pairs among the K top-ranked experts, pair accumulators in registers.
+// `ref` (optional) is the token's target row F_ref[h] in fp32; without it the target is the
+// unpruned output built from the two top-ranked experts.
 template <int K>
 __device__ __forceinline__ void pair_errors_fast(const bf16* __restrict__ Yt, int h,
                                                  const int* order, const float* l, int lane,
-                                                 float* s_err /* [16*16] */) {
+                                                 float* s_err /* [16*16] */,
+                                                 const float* __restrict__ ref) {
   constexpr int NP = K * (K - 1) / 2;
   float wa[NP], wb[NP], err[NP];
   {
@@ -57,9 +60,16 @@ __device__ __forceinline__ void pair_errors_fast(const bf16* __restrict__ Yt, in
     float y[K][8];
 #pragma unroll
     for (int i = 0; i < K; ++i) unpack8f(__ldg(rows[i] + v), y[i]);
+    float fr[8];
+    if (ref) {
+      const float4 r0 = __ldg(reinterpret_cast<const float4*>(ref) + 2 * v);
+      const float4 r1 = __ldg(reinterpret_cast<const float4*>(ref) + 2 * v + 1);
+      fr[0] = r0.x; fr[1] = r0.y; fr[2] = r0.z; fr[3] = r0.w;
+      fr[4] = r1.x; fr[5] = r1.y; fr[6] = r1.z; fr[7] = r1.w;
+    }
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-      const float F = fmaf(wb[0], y[1][k], wa[0] * y[0][k]);
+      const float F = ref ? fr[k] : fmaf(wb[0], y[1][k], wa[0] * y[0][k]);
       int p = 0;
 #pragma unroll
       for (int i = 0; i < K; ++i)
@@ -85,7 +95,7 @@ __device__ __forceinline__ void pair_errors_fast(const bf16* __restrict__ Yt, in
 // The same for any K, one pair at a time (rows are re-read from cache).
 __device__ __forceinline__ void pair_errors_generic(const bf16* __restrict__ Yt, int h, int K,
                                                     const int* order, const float* l, int lane,
-                                                    float* s_err) {
+                                                    float* s_err, const float* __restrict__ ref) {
   float w0, w1;
   pair_weights(l[order[0]], l[order[1]], w0, w1);
   const uint4* r0 = reinterpret_cast<const uint4*>(Yt + (size_t)order[0] * h);
@@ -105,7 +115,7 @@ __device__ __forceinline__ void pair_errors_generic(const bf16* __restrict__ Yt,
         unpack8f(__ldg(rj + v), yj);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          const float F = fmaf(w1, y1[k], w0 * y0[k]);
+          const float F = ref ? ref[8 * v + k] : fmaf(w1, y1[k], w0 * y0[k]);
           const float d = fmaf(wb, yj[k], wa * yi[k]) - F;
           e = fmaf(d, d, e);
         }
@@ -119,7 +129,7 @@ __device__ __forceinline__ void pair_errors_generic(const bf16* __restrict__ Yt,
 __global__ void __launch_bounds__(128)
 enumerate_kernel(const float* __restrict__ logits, const bf16* __restrict__ Yall, int T, int E,
                  int r, int h, const uint32_t* __restrict__ subsets, int nC,
-                 float* __restrict__ partial) {
+                 float* __restrict__ partial, const float* __restrict__ Fref) {
   extern __shared__ float s_dyn[];
   const int nwarps = blockDim.x >> 5;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -153,13 +163,14 @@ enumerate_kernel(const float* __restrict__ logits, const bf16* __restrict__ Yall
     }
     __syncwarp();
     const bf16* Yt = Yall + (size_t)t * E * h;
+    const float* ref = Fref ? Fref + (size_t)t * h : nullptr;
     switch (K) {
-      case 2: pair_errors_fast<2>(Yt, h, s_order, s_l, lane, s_err); break;
-      case 3: pair_errors_fast<3>(Yt, h, s_order, s_l, lane, s_err); break;
-      case 4: pair_errors_fast<4>(Yt, h, s_order, s_l, lane, s_err); break;
-      case 5: pair_errors_fast<5>(Yt, h, s_order, s_l, lane, s_err); break;
-      case 6: pair_errors_fast<6>(Yt, h, s_order, s_l, lane, s_err); break;
-      default: pair_errors_generic(Yt, h, K, s_order, s_l, lane, s_err); break;
+      case 2: pair_errors_fast<2>(Yt, h, s_order, s_l, lane, s_err, ref); break;
+      case 3: pair_errors_fast<3>(Yt, h, s_order, s_l, lane, s_err, ref); break;
+      case 4: pair_errors_fast<4>(Yt, h, s_order, s_l, lane, s_err, ref); break;
+      case 5: pair_errors_fast<5>(Yt, h, s_order, s_l, lane, s_err, ref); break;
+      case 6: pair_errors_fast<6>(Yt, h, s_order, s_l, lane, s_err, ref); break;
+      default: pair_errors_generic(Yt, h, K, s_order, s_l, lane, s_err, ref); break;
     }
     __syncwarp();
     for (int s = lane; s < nC; s += 32) {
@@ -206,7 +217,7 @@ int enumerate_num_blocks(int T, int nC) {
 
 cudaError_t launch_enumerate(const float* logits, const bf16* Yall, int T, int E, int r, int h,
                              const uint32_t* subsets, int nC, float* partial, double* loss_sq,
-                             float* losses, cudaStream_t st) {
+                             float* losses, const float* Fref, cudaStream_t st) {
   const int nw = warps_for(nC);
   const int nblk = enumerate_num_blocks(T, nC);
   const size_t smem = ((size_t)nw * nC + (size_t)nw * kMaxE * kMaxE + 2 * (size_t)nw * kMaxE) * 4;
@@ -218,7 +229,7 @@ cudaError_t launch_enumerate(const float* logits, const bf16* Yall, int T, int E
     attr_set = true;
   }
   if (smem > 96 * 1024) return cudaErrorInvalidValue;
-  enumerate_kernel<<<nblk, nw * 32, smem, st>>>(logits, Yall, T, E, r, h, subsets, nC, partial);
+  enumerate_kernel<<<nblk, nw * 32, smem, st>>>(logits, Yall, T, E, r, h, subsets, nC, partial, Fref);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   reduce_partials_kernel<<<(nC + 127) / 128, 128, 0, st>>>(partial, nblk, nC, loss_sq, losses);

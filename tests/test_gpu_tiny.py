@@ -283,3 +283,23 @@ def test_coselection_and_frequency_baseline(setup):
     assert np.array(pruned.coselection(x.to(DEV)))[6:, :].sum() == 0
     pruned.close()
     layer.close()
+
+
+@pytest.mark.parametrize("r", [6, 4])
+def test_progressive_search_matches_oracle(setup, r):
+    host, dev = setup
+    T = 333
+    x = synth.make_tokens(T, H, seed=0)       # states of the unpruned stack
+    xp = synth.make_tokens(T, H, seed=5)      # states that went through pruned layers
+    layer = make_layer(dev)
+    F_ref = layer.forward(x.to(DEV), 0.0).float().contiguous()   # cached unpruned output (bf16 -> fp32)
+    ora = O.prune_search_progressive(synth.bf16_bits(xp), host["Wg"], host["W1"], host["W3"], host["W2"],
+                                     F_ref.cpu().numpy(), r)
+    losses, best = layer.prune_search_progressive(xp.to(DEV), F_ref, r)
+    P.check_search(losses, best, ora)
+    # identical inputs on both sides: the layer-wise losses up to the bf16 rounding of the cached target
+    lw, _ = layer.prune_search(x.to(DEV), r)
+    pg, _ = layer.prune_search_progressive(x.to(DEV), F_ref, r)
+    fn = float(F_ref.double().norm())
+    assert np.abs(np.array(pg) - np.array(lw)).max() <= 2 ** -8 * fn
+    layer.close()

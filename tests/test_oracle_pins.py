@@ -342,3 +342,52 @@ def test_coselection_counts_and_frequency_subset(cfg0, dense):
     c = np.zeros((4, 4), np.int64)
     c[0, 1] = c[2, 3] = 5
     assert O.frequency_subset(c, 2) == 0b0011
+
+
+# ----------------------------------------------------------- progressive search
+
+def _unpruned_output(c, Y_rounded):
+    r = O.route(c["x"], c["Wg"], FULL, 0.0)
+    t = np.arange(len(c["x"]))
+    return (r["wn"][:, 0:1].astype(np.float64) * Y_rounded[t, r["idx"][:, 0]]
+            + r["wn"][:, 1:2].astype(np.float64) * Y_rounded[t, r["idx"][:, 1]])
+
+
+def test_progressive_search_reduces_to_layerwise_on_identical_inputs(cfg0):
+    """With x_p = x and F_ref = F(x) the progressive loss is the layer-wise loss of Eq. 3."""
+    Y = O.all_experts(cfg0["x"], cfg0["W1"], cfg0["W3"], cfg0["W2"], round_bf16=True)
+    F = _unpruned_output(cfg0, Y)
+    lw = search(cfg0, 6, True)
+    pg = O.prune_search_progressive(cfg0["x"], cfg0["Wg"], cfg0["W1"], cfg0["W3"], cfg0["W2"],
+                                    F.astype(np.float32), 6)
+    # F_ref is stored in fp32: one rounding of relative size 2^-24 on every element
+    tol = 2e-7 * np.linalg.norm(F)
+    assert np.abs(pg["losses"] - lw["losses"]).max() <= tol + 1e-6 * lw["losses"].max()
+    assert pg["best_subset"] == lw["best_subset"]
+
+
+def test_progressive_search_matches_dense_restatement(cfg0, dense):
+    """Different inputs on the two sides: pruned layer on x_p (dense numpy), target from x."""
+    Yx = D.round_bf16(dense["Y"])
+    F_ref = _unpruned_output(cfg0, Yx).astype(np.float32)
+    xp = synth.bf16_bits(synth.make_tokens(T, H, seed=5))
+    lp = D.logits(xp, cfg0["Wg"])
+    Yp = D.round_bf16(D.all_experts(xp, cfg0["W1"], cfg0["W3"], cfg0["W2"]))
+    pg = O.prune_search_progressive(xp, cfg0["Wg"], cfg0["W1"], cfg0["W3"], cfg0["W2"], F_ref, 6)
+    t = np.arange(T)
+    for ci in (0, 9, 27):
+        e0, e1, _, _ = D.top2(lp, int(pg["subsets"][ci]))
+        d = lp[t, e1] - lp[t, e0]
+        Fp = (1 / (1 + np.exp(d)))[:, None] * Yp[t, e0] + (1 / (1 + np.exp(-d)))[:, None] * Yp[t, e1]
+        want = np.linalg.norm(Fp - F_ref.astype(np.float64))
+        assert abs(pg["losses"][ci] - want) < 1e-5 * want
+    # additive over token chunks, and a zero target gives the norm of the pruned output itself
+    a = O.prune_search_progressive(xp[:90], cfg0["Wg"], cfg0["W1"], cfg0["W3"], cfg0["W2"], F_ref[:90], 6)
+    b = O.prune_search_progressive(xp[90:], cfg0["Wg"], cfg0["W1"], cfg0["W3"], cfg0["W2"], F_ref[90:], 6)
+    np.testing.assert_allclose(a["loss_sq"] + b["loss_sq"], pg["loss_sq"], rtol=1e-12)
+    z = O.prune_search_progressive(xp, cfg0["Wg"], cfg0["W1"], cfg0["W3"], cfg0["W2"],
+                                   np.zeros((T, H), np.float32), 8)
+    e0, e1, _, _ = D.top2(lp, FULL)
+    d = lp[t, e1] - lp[t, e0]
+    Ffull = (1 / (1 + np.exp(d)))[:, None] * Yp[t, e0] + (1 / (1 + np.exp(-d)))[:, None] * Yp[t, e1]
+    assert abs(z["losses"][0] - np.linalg.norm(Ffull)) < 1e-5 * np.linalg.norm(Ffull)
