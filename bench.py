@@ -491,6 +491,8 @@ def run_stack(a):
             mask = 0xFF
         else:
             full = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, 0xFF)
+            if layers:
+                full.share_scratch(layers[0])  # one set of search scratch for the whole stack
             torch.cuda.synchronize(dev)
             t0 = time.perf_counter()
             if state_p is None:

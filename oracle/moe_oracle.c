@@ -303,6 +303,91 @@ int oracle_moe_forward(const uint16_t *x, const uint16_t *Wg, const uint16_t *W1
   return 0;
 }
 
+/* ------------------------------------------------------- top-k generalisation */
+
+/* Routing of one token in the general top-k setting (App. A.2).  e_0..e_{k-1} are the kept
+ * experts with the k largest routing weights (ties to the lower index), p_m = exp(l_em - l_e0)
+ * their softmax numerators (the denominator cancels everywhere).  Dynamic skipping keeps the
+ * top-i* experts with
+ *     i* = min i in 1..k  such that  sum_{m=i+1..k} w_m <= beta * sum_{m=1..k} w_m
+ * (the paper's 1-based m), and the output is renormalised over those i* experts.
+ * fp32 order of the sums, the same on the CUDA side: the total over the k experts in
+ * ascending m; the tails accumulated from the smallest weight upwards; the kept mass in
+ * ascending m. */
+static void route_token_topk(const float *l, int E, uint32_t kept, int k, float beta, int32_t *idx,
+                             float *wn, int *n_active, float *tail_frac) {
+  uint32_t left = kept;
+  float p[ORACLE_MAX_E];
+  for (int m = 0; m < k; ++m) {
+    int best = -1;
+    for (int e = 0; e < E; ++e)
+      if (((left >> e) & 1u) && (best < 0 || l[e] > l[best])) best = e;
+    idx[m] = best;
+    left &= ~(1u << best);
+    p[m] = expf(l[best] - l[idx[0]]);
+  }
+  float total = 0.0f;
+  for (int m = 0; m < k; ++m) total += p[m];
+  float tail[ORACLE_MAX_E + 1];
+  tail[k] = 0.0f;
+  for (int m = k - 1; m >= 1; --m) tail[m] = tail[m + 1] + p[m];
+  int istar = k;
+  for (int i = 1; i <= k; ++i)
+    if (tail[i] <= beta * total) { istar = i; break; }
+  float keep = 0.0f;
+  for (int m = 0; m < istar; ++m) keep += p[m];
+  for (int m = 0; m < k; ++m) wn[m] = m < istar ? p[m] / keep : 0.0f;
+  *n_active = istar;
+  if (tail_frac) *tail_frac = tail[istar] / total;
+}
+
+/* Layer forward with top-k routing and the generalised skipping rule above.
+ * idx[T][k], wn[T][k] (0 for skipped experts), n_active[T]; z64/y as in oracle_moe_forward;
+ * tail_frac[T] = skipped mass / total mass of the k selected (0 when nothing is skipped). */
+int oracle_moe_forward_topk(const uint16_t *x, const uint16_t *Wg, const uint16_t *W1,
+                            const uint16_t *W3, const uint16_t *W2, int T, int h, int f, int E,
+                            uint32_t kept_mask, int k, float beta, uint16_t *y, double *z64,
+                            int32_t *idx, float *wn, int32_t *n_active, float *tail_frac,
+                            float *logits) {
+  if (E < 2 || E > ORACLE_MAX_E || k < 1 || popcount32(kept_mask & ((1u << E) - 1u)) < k) return -1;
+#pragma omp parallel
+  {
+    float *a = (float *)malloc(sizeof(float) * (size_t)f);
+    double *o = (double *)malloc(sizeof(double) * (size_t)h);
+    double *z = (double *)malloc(sizeof(double) * (size_t)h);
+#pragma omp for schedule(dynamic, 1)
+    for (int t = 0; t < T; ++t) {
+      const uint16_t *xt = x + (size_t)t * h;
+      float l[ORACLE_MAX_E], w[ORACLE_MAX_E], tf;
+      int32_t id[ORACLE_MAX_E];
+      int na;
+      router_logits(xt, Wg, h, E, l);
+      route_token_topk(l, E, kept_mask, k, beta, id, w, &na, &tf);
+      for (int i = 0; i < h; ++i) z[i] = 0.0;
+      for (int m = 0; m < na; ++m) {
+        expert_ffn(xt, W1 + (size_t)id[m] * f * h, W3 + (size_t)id[m] * f * h,
+                   W2 + (size_t)id[m] * h * f, h, f, o, a);
+        for (int i = 0; i < h; ++i) z[i] += (double)w[m] * o[i];
+      }
+      for (int i = 0; i < h; ++i) {
+        if (z64) z64[(size_t)t * h + i] = z[i];
+        if (y) y[(size_t)t * h + i] = f32_to_bf16((float)z[i]);
+      }
+      for (int m = 0; m < k; ++m) {
+        if (idx) idx[(size_t)t * k + m] = id[m];
+        if (wn) wn[(size_t)t * k + m] = w[m];
+      }
+      if (n_active) n_active[t] = na;
+      if (tail_frac) tail_frac[t] = tf;
+      if (logits) memcpy(logits + (size_t)t * E, l, sizeof(float) * (size_t)E);
+    }
+    free(a);
+    free(o);
+    free(z);
+  }
+  return 0;
+}
+
 /* ------------------------------------------------------------------ beta */
 
 static int cmp_float(const void *a, const void *b) {

@@ -175,6 +175,33 @@ def frequency_subset(counts, r: int) -> int:
     return int(fn(_p(counts, _i64p), E, r))
 
 
+def moe_forward_topk(x, Wg, W1, W3, W2, kept_mask: int, k: int, beta: float):
+    """Top-k layer forward with the generalised skipping rule.  Returns dict(y, z, idx[T,k],
+    wn[T,k], n_active[T], tail_frac[T], logits[T,E])."""
+    x = _u16(x)
+    T, h = x.shape
+    Wg = _u16(Wg)
+    E = Wg.shape[0]
+    W1 = _u16(W1)
+    f = W1.shape[1]
+    W3 = _u16(W3, (E, f, h))
+    W2 = _u16(W2, (E, h, f))
+    out = dict(
+        y=np.zeros((T, h), np.uint16), z=np.zeros((T, h), np.float64),
+        idx=np.zeros((T, k), np.int32), wn=np.zeros((T, k), np.float32),
+        n_active=np.zeros((T,), np.int32), tail_frac=np.zeros((T,), np.float32),
+        logits=np.zeros((T, E), np.float32),
+    )
+    rc = lib().oracle_moe_forward_topk(
+        _p(x, _u16p), _p(Wg, _u16p), _p(W1, _u16p), _p(W3, _u16p), _p(W2, _u16p), T, h, f, E,
+        ctypes.c_uint32(kept_mask), k, ctypes.c_float(beta), _p(out["y"], _u16p), _p(out["z"], _f64p),
+        _p(out["idx"], _i32p), _p(out["wn"], _f32p), _p(out["n_active"], _i32p),
+        _p(out["tail_frac"], _f32p), _p(out["logits"], _f32p))
+    if rc:
+        raise ValueError("oracle_moe_forward_topk: invalid arguments")
+    return out
+
+
 def beta_median(ratio) -> float:
     ratio = np.ascontiguousarray(ratio, dtype=np.float32)
     b = ctypes.c_float(0)

@@ -391,3 +391,98 @@ def test_progressive_search_matches_dense_restatement(cfg0, dense):
     d = lp[t, e1] - lp[t, e0]
     Ffull = (1 / (1 + np.exp(d)))[:, None] * Yp[t, e0] + (1 / (1 + np.exp(-d)))[:, None] * Yp[t, e1]
     assert abs(z["losses"][0] - np.linalg.norm(Ffull)) < 1e-5 * np.linalg.norm(Ffull)
+
+
+# ------------------------------------------------------- generalised top-k skipping
+
+@pytest.fixture(scope="module")
+def cfg16():
+    h, f, E_, T_ = 64, 128, 16, 200
+    W = synth.make_layer_weights(h, f, E_, seed=7)
+    x = synth.make_tokens(T_, h, seed=8)
+    b = synth.bf16_bits
+    c = dict(x=b(x), Wg=b(W.W_gate), W1=b(W.W1), W3=b(W.W3), W2=b(W.W2))
+    return c, D.logits(c["x"], c["Wg"]), D.all_experts(c["x"], c["W1"], c["W3"], c["W2"])
+
+
+def fwdk(c, kept, k, beta):
+    return O.moe_forward_topk(c["x"], c["Wg"], c["W1"], c["W3"], c["W2"], kept, k, beta)
+
+
+@pytest.mark.parametrize("k", [1, 2, 4])
+def test_topk_without_skipping_is_textbook_topk(cfg16, k):
+    """beta = 0: App. A.2's z = sum_{m<=k} w_m f_m / sum_{m<=k} w_m, as dense then mask."""
+    c, l, Y = cfg16
+    kept = 0xFFFF
+    out = fwdk(c, kept, k, 0.0)
+    Tn = l.shape[0]
+    order = np.argsort(-l, axis=1, kind="stable")
+    srt = np.take_along_axis(l, order, 1)
+    ok = (np.diff(-srt[:, :k + 1], axis=1) > 1e-3).all(1)
+    assert ok.sum() > 0.8 * Tn
+    assert np.array_equal(out["idx"][ok], order[ok, :k])
+    assert (out["n_active"] == k).all()
+    sm = np.exp(l - l.max(1, keepdims=True))
+    mask = np.zeros_like(sm)
+    np.put_along_axis(mask, order[:, :k], 1.0, axis=1)
+    wt = sm * mask
+    wt /= wt.sum(1, keepdims=True)
+    z = np.einsum("te,teh->th", wt, Y)
+    assert np.abs(out["z"][ok] - z[ok]).max() < 3e-6 * np.abs(z).max()
+    np.testing.assert_allclose(out["wn"].sum(1), 1.0, rtol=1e-6)
+
+
+def test_topk_skipping_rule_bound_and_monotonicity(cfg16):
+    """i* is the smallest i whose skipped mass is <= beta of the selected mass; the output
+    error obeys the appendix' bound L <= (skipped mass / selected mass) * max ||f_m - f_n||."""
+    c, l, Y = cfg16
+    kept, k = 0xFFFF, 4
+    base = fwdk(c, kept, k, 0.0)
+    t = np.arange(l.shape[0])
+    prev = np.full(l.shape[0], k)
+    for beta in (0.05, 0.2, 0.5, 0.9, 1.0):
+        out = fwdk(c, kept, k, beta)
+        na = out["n_active"]
+        assert (na <= prev).all() and (na >= 1).all()
+        prev = na
+        assert np.array_equal(out["idx"], base["idx"])
+        # the rule, re-evaluated in fp64 from the dense logits (away from the threshold)
+        sel = np.take_along_axis(l, base["idx"].astype(np.int64), 1)
+        p = np.exp(sel - sel[:, :1])
+        tot = p.sum(1)
+        tails = np.stack([p[:, i:].sum(1) for i in range(1, k + 1)], 1)  # i = 1..k
+        want = 1 + (tails > beta * tot[:, None]).sum(1)
+        clear = (np.abs(tails / tot[:, None] - beta) > 1e-5).all(1)
+        assert np.array_equal(na[clear], want[clear])
+        np.testing.assert_allclose(out["tail_frac"], tails[t, na - 1] / tot, rtol=1e-5, atol=1e-7)
+        assert (out["tail_frac"] <= beta + 1e-6).all()
+        # weights renormalised over the survivors, zero for the skipped ones
+        assert (out["wn"][t[:, None], np.arange(k)[None, :]] * (np.arange(k)[None, :] >= na[:, None]) == 0).all()
+        np.testing.assert_allclose(out["wn"].sum(1), 1.0, rtol=1e-6)
+        # the paper's bound on the reconstruction error
+        f_sel = Y[t[:, None], base["idx"]]                         # [T, k, h]
+        dmax = np.max(np.linalg.norm(f_sel[:, :, None, :] - f_sel[:, None, :, :], axis=3), axis=(1, 2))
+        err = np.linalg.norm(out["z"] - base["z"], axis=1)
+        assert (err <= out["tail_frac"] * dmax * (1 + 1e-6) + 1e-12).all()
+    assert (fwdk(c, kept, k, 1.0)["n_active"] == 1).all()          # beta >= 1 degenerates to top-1
+
+
+def test_top2_generalised_rule_is_the_pairwise_rule_with_rescaled_beta(cfg0):
+    """For k = 2, w_2 <= b (w_1 + w_2) is w_2 <= b/(1-b) w_1: the two forms of the paper agree."""
+    bg = 0.3
+    g = O.moe_forward_topk(cfg0["x"], cfg0["Wg"], cfg0["W1"], cfg0["W3"], cfg0["W2"], FULL, 2, bg)
+    pw = fwd(cfg0, beta=bg / (1 - bg))
+    away = np.abs(pw["ratio"] - bg / (1 - bg)) > 1e-5
+    assert np.array_equal((g["n_active"] == 1)[away], pw["skipped"].astype(bool)[away])
+    assert np.array_equal(g["idx"], pw["idx"])
+    same = (g["n_active"] == 1) == pw["skipped"].astype(bool)
+    np.testing.assert_allclose(g["z"][same], pw["z"][same], rtol=1e-6, atol=1e-9)
+
+
+def test_topk_pruned_experts_are_never_selected(cfg16):
+    c, l, Y = cfg16
+    kept = 0b1010110011110101
+    out = fwdk(c, kept, 4, 0.3)
+    assert all((kept >> int(e)) & 1 for e in out["idx"].ravel())
+    with pytest.raises(ValueError):
+        fwdk(c, 0b111, 4, 0.0)
