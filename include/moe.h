@@ -99,6 +99,23 @@ int moe_forward_residual(moe_layer_t* layer, const void* x, int T, float beta,
                          const void* residual, void* y, void* routing_stats);
 
 /*
+ * Layer forward in the general top-k setting with the generalised skipping
+ * rule of App. A.2: e_0..e_{k-1} are the kept experts with the k largest routing
+ * weights; the top i* of them run, where
+ *     i* = min i  such that  sum_{m=i+1..k} w_m <= beta * sum_{m=1..k} w_m,
+ * and the output is renormalised over those i*:
+ *     z = sum_{m<=i*} w_m E_m(x) / sum_{m<=i*} w_m.
+ * beta = 0 keeps all k, beta >= 1 keeps only the first.  (For k = 2 this is the
+ * rule of moe_forward with beta/(1-beta) in place of beta and "<=" for "<".)
+ * 1 <= k <= min(kept experts, 8).  Optional device outputs: idx_out [T][k] int32
+ * original expert ids in order of decreasing weight, wn_out [T][k] the weights
+ * applied (0 for skipped experts), n_active_out [T] int32 = i*.  x, y as in
+ * moe_forward.  Asynchronous.
+ */
+int moe_forward_topk(moe_layer_t* layer, const void* x, int T, int k, float beta, void* y,
+                     int32_t* idx_out, float* wn_out, int32_t* n_active_out);
+
+/*
  * moe_forward with HOST buffers: copies x_host to the device, runs the layer,
  * copies y back and waits for it.  x_host/y_host [T][h] bf16; pinned memory
  * makes the copies asynchronous to the host but is not required.

@@ -54,6 +54,7 @@ def load_library(path: str | None = None):
     lib.moe_forward.argtypes = [vp, vp, ci, cf, vp, vp]
     lib.moe_forward_residual.argtypes = [vp, vp, ci, cf, vp, vp, vp]
     lib.moe_forward_host.argtypes = [vp, vp, ci, cf, vp]
+    lib.moe_forward_topk.argtypes = [vp, vp, ci, ci, cf, vp, vp, vp, vp]
     lib.moe_routing_stats_layout.restype = ctypes.c_size_t
     lib.moe_routing_stats_layout.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_size_t)]
     lib.moe_routing_stats_bytes.restype = ctypes.c_size_t
@@ -183,6 +184,23 @@ class MoeLayer:
             _check(lib.moe_forward_residual(self._h, x.data_ptr(), T, beta, residual.data_ptr(),
                                             y.data_ptr(), sp))
         return y
+
+    def forward_topk(self, x, k: int, beta: float = 0.0, y=None, record: bool = False):
+        """``moe_forward_topk``; with ``record`` also returns (idx[T,k] i32, wn[T,k] f32, n_active[T] i32)."""
+        T = x.shape[0]
+        _dev_bf16(x, (T, self.h))
+        if y is None:
+            y = torch.empty_like(x)
+        idx = wn = na = None
+        if record:
+            idx = torch.zeros((T, max(k, 1)), dtype=torch.int32, device=x.device)
+            wn = torch.zeros((T, max(k, 1)), dtype=torch.float32, device=x.device)
+            na = torch.zeros((T,), dtype=torch.int32, device=x.device)
+        _check(load_library().moe_forward_topk(
+            self._h, x.data_ptr(), T, k, beta, y.data_ptr(),
+            idx.data_ptr() if record else None, wn.data_ptr() if record else None,
+            na.data_ptr() if record else None))
+        return (y, idx, wn, na) if record else y
 
     def forward_host(self, x_host: torch.Tensor, beta: float, y_host: torch.Tensor):
         """``moe_forward_host``: x_host, y_host are host bf16 tensors (pinned or not)."""

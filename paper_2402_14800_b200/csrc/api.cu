@@ -66,6 +66,8 @@ struct Workspace {
   Buf s_logits, s_yall, s_act, s_subsets, s_partial, s_loss_sq, s_losses, s_xpad, s_meta;
   // host staging and stack scratch
   Buf hx, hy, xn, cosel;
+  // general top-k path
+  Buf k_idx, k_wn, k_pos, k_nact;
 };
 
 int moe::set_error(int code, const char* fmt, ...) {
@@ -149,9 +151,9 @@ int ensure_route(moe_layer* L, int T) {
 }
 
 inline bool decode_mode(int T) { return T <= kDecodeMaxT; }
-inline int rows_for(const moe_layer* L, int T) {
+inline int rows_for(const moe_layer* L, int T, int k = 2) {
   const int pad = decode_mode(T) ? 16 : kTileRows;
-  return (int)align_up((size_t)2 * T + (size_t)L->r * pad, 16);
+  return (int)align_up((size_t)k * T + (size_t)L->r * pad, 16);
 }
 inline int ksplit_for(const moe_layer* L) {
   const int KB = (L->f + 63) / 64;
@@ -165,9 +167,9 @@ int build_token_maps(GemmMaps& m, const void* base, uint64_t inner, uint64_t row
   return MOE_OK;
 }
 
-int ensure_gemm(moe_layer* L, int T) {
+int ensure_gemm(moe_layer* L, int T, int k = 2) {
   // capacity in rows: large enough for this T in its mode, at least 256 (TMA boxes)
-  int need = (int)align_up((size_t)rows_for(L, T), kTileRows) + kTileRows;
+  int need = (int)align_up((size_t)rows_for(L, T, k), kTileRows) + kTileRows;
   if (need < 256) need = 256;
   size_t need_O = (size_t)need * L->h * (decode_mode(T) ? ksplit_for(L) : 1);
   if (need <= L->ws->cap_rows && need_O * 4 <= L->ws->O.bytes && L->ws->map_h == L->h &&
@@ -428,7 +430,7 @@ void moe_layer_destroy(moe_layer_t* L) {
   Buf* bufs[] = {&L->own.idx, &L->own.wn, &L->own.ratio, &L->own.skipped, &L->own.blk_hist, &L->own.blk_base, &L->own.pair_pos,
                  &L->own.meta, &L->own.status, &L->own.sel, &L->own.row_token, &L->own.xperm, &L->own.act, &L->own.O, &L->own.tail,
                  &L->own.s_logits, &L->own.s_yall, &L->own.s_act, &L->own.s_subsets, &L->own.s_partial, &L->own.s_loss_sq,
-                 &L->own.s_losses, &L->own.s_xpad, &L->own.s_meta, &L->own.hx, &L->own.hy, &L->own.xn, &L->own.cosel};
+                 &L->own.s_losses, &L->own.s_xpad, &L->own.s_meta, &L->own.hx, &L->own.hy, &L->own.xn, &L->own.cosel, &L->own.k_idx, &L->own.k_wn, &L->own.k_pos, &L->own.k_nact};
   for (Buf* b : bufs) release(L, *b);
   for (cudaEvent_t e : L->prof_ev) cudaEventDestroy(e);
   if (L->Wg) cudaFree(L->Wg);
@@ -453,6 +455,66 @@ int moe_forward(moe_layer_t* L, const void* x, int T, float beta, void* y, void*
 int moe_forward_residual(moe_layer_t* L, const void* x, int T, float beta, const void* residual,
                          void* y, void* routing_stats) {
   return forward_impl(L, x, T, beta, residual, y, routing_stats);
+}
+
+int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, void* y,
+                     int32_t* idx_out, float* wn_out, int32_t* n_active_out) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
+  if (k < 1 || k > L->r || k > 8) return fail(MOE_ERR_INVALID_ARG, "k = %d outside 1..min(kept experts, 8)", k);
+  if (T == 0) return MOE_OK;
+  if (!x || !y || x == y) return fail(MOE_ERR_INVALID_ARG, "x and y must be distinct and non-NULL");
+  if (!aligned16(x) || !aligned16(y)) return fail(MOE_ERR_INVALID_ARG, "x and y must be 16-byte aligned");
+  if (!(beta >= 0.f)) return fail(MOE_ERR_INVALID_ARG, "beta must be >= 0");
+  int rc;
+  if ((rc = ensure_route(L, T))) return rc;
+  if ((rc = ensure_gemm(L, T, k))) return rc;
+  Workspace& W = *L->ws;
+  if ((rc = grow(L, W.k_idx, (size_t)T * k * 4))) return rc;
+  if ((rc = grow(L, W.k_wn, (size_t)T * k * 4))) return rc;
+  if ((rc = grow(L, W.k_pos, (size_t)T * k * 4))) return rc;
+  if ((rc = grow(L, W.k_nact, (size_t)T * 4))) return rc;
+  cudaStream_t st = L->stream;
+  const bool dec = decode_mode(T);
+  const int nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
+  const int rows_cap = rows_for(L, T, k);
+  Meta* meta = (Meta*)W.meta.p;
+  int32_t* idx = (int32_t*)W.k_idx.p;
+  int32_t* nact = (int32_t*)W.k_nact.p;
+  CUDA_TRY(launch_router_topk((const bf16*)x, L->Wg, T, L->h, L->r, k, beta, L->kept, idx,
+                              (float*)W.k_wn.p, nact, idx_out, wn_out, n_active_out, st));
+  CUDA_TRY(launch_count_topk(idx, nact, T, k, (int32_t*)W.blk_hist.p, st));
+  CUDA_TRY(launch_scan((int32_t*)W.blk_hist.p, nblk, L->r, dec ? 16 : kTileRows, (int32_t*)W.blk_base.p,
+                       meta, nullptr, nullptr, nullptr, L->kept, L->E, st));
+  CUDA_TRY(cudaMemsetAsync(W.row_token.p, 0xff, (size_t)rows_cap * 4, st));
+  CUDA_TRY(launch_scatter_topk(idx, nact, (int32_t*)W.blk_base.p, meta, T, k, (int32_t*)W.k_pos.p,
+                               (int32_t*)W.row_token.p, st));
+  CUDA_TRY(launch_gather((const bf16*)x, (int32_t*)W.row_token.p, meta, L->h, rows_cap,
+                         (bf16*)W.xperm.p, st));
+  GemmArgs gu, dn;
+  memset(&gu, 0, sizeof(gu));
+  memset(&dn, 0, sizeof(dn));
+  gu.a_off_mul = 1; gu.out_off_mul = 1; gu.out_ld = L->f; gu.out = W.act.p;
+  dn.a_off_mul = 1; dn.out_off_mul = 1; dn.out_ld = L->h; dn.out = W.O.p;
+  const bool wm = dec && !L->debug_simt;
+  if (wm) { gu.tail = (float*)W.tail.p; dn.tail = (float*)W.tail.p; }
+  const int ksplit = wm ? ksplit_for(L) : 1;
+  const size_t split_stride = (size_t)rows_cap * L->h;
+  dn.split_stride = (long long)split_stride;
+  GemmMaps m_gu, m_dn;
+  m_gu.w = wm ? L->w13_128 : L->w13_256;
+  m_dn.w = wm ? L->w2_128 : L->w2_256;
+  memcpy(m_gu.t, W.tok_x, sizeof(m_gu.t));
+  memcpy(m_dn.t, W.tok_act, sizeof(m_dn.t));
+  const bool prof_saved = L->prof;
+  L->prof = false;
+  rc = run_expert_gemms(L, meta, wm, m_gu, m_dn, gu, dn, kOutF32, (const bf16*)W.xperm.p,
+                        (const bf16*)W.act.p, rows_cap);
+  L->prof = prof_saved;
+  if (rc) return rc;
+  CUDA_TRY(launch_combine_topk((const float*)W.O.p, ksplit, split_stride, (int32_t*)W.k_pos.p,
+                               (float*)W.k_wn.p, k, T, L->h, (bf16*)y, st));
+  return MOE_OK;
 }
 
 int moe_forward_host(moe_layer_t* L, const void* x_host, int T, float beta, void* y_host) {

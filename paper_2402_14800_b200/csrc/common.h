@@ -103,6 +103,18 @@ cudaError_t launch_gather(const bf16* x, const int32_t* row_token, const Meta* m
 cudaError_t launch_combine(const float* O, int ksplit, size_t split_stride, const int32_t* pair_pos,
                            const float* wn, const bf16* residual, int T, int h, bf16* y,
                            cudaStream_t st);
+// general top-k path (k slots per token instead of two)
+cudaError_t launch_router_topk(const bf16* x, const bf16* Wg, int T, int h, int r, int k, float beta,
+                               const KeptIds& kept, int32_t* idx, float* wn, int32_t* nact,
+                               int32_t* u_idx, float* u_wn, int32_t* u_nact, cudaStream_t st);
+cudaError_t launch_count_topk(const int32_t* idx, const int32_t* nact, int T, int k,
+                              int32_t* blk_hist, cudaStream_t st);
+cudaError_t launch_scatter_topk(const int32_t* idx, const int32_t* nact, const int32_t* blk_base,
+                                const Meta* meta, int T, int k, int32_t* pair_pos,
+                                int32_t* row_token, cudaStream_t st);
+cudaError_t launch_combine_topk(const float* O, int ksplit, size_t split_stride,
+                                const int32_t* pair_pos, const float* wn, int k, int T, int h,
+                                bf16* y, cudaStream_t st);
 cudaError_t launch_coselection(const int32_t* idx, int T, int E, const KeptIds& kept, int32_t* counts,
                                cudaStream_t st);
 cudaError_t launch_rmsnorm(const bf16* x, int T, int h, float eps, bf16* out, cudaStream_t st);

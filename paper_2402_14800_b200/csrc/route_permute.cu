@@ -446,6 +446,165 @@ combine_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
   }
 }
 
+
+// ------------------------------------------------------------------ general top-k path
+
+// Top-k routing with the generalised skipping rule of App. A.2, one block per token:
+//   e_0..e_{k-1} = kept experts with the k largest logits (ties to the lower index),
+//   p_m = exp(l_em - l_e0);  keep the top i* = min i : sum_{m>i} p_m <= beta * sum_{m<=k} p_m;
+//   weights p_m / sum_{m<=i*} p_m.  The fp32 summation orders are fixed: total ascending in m,
+//   tails from the smallest upwards, kept mass ascending in m.
+__global__ void __launch_bounds__(256)
+router_topk_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, int h, int r,
+                   int k, float beta, KeptIds kept, int32_t* __restrict__ idx,
+                   float* __restrict__ wn, int32_t* __restrict__ nact, int32_t* u_idx, float* u_wn,
+                   int32_t* u_nact) {
+  __shared__ float s_part[8][kMaxE];
+  const int t = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nvec = h >> 3;
+  float acc[kMaxE];
+#pragma unroll
+  for (int c = 0; c < kMaxE; ++c) acc[c] = 0.f;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)t * h);
+  for (int v = threadIdx.x; v < nvec; v += 256) {
+    float xf[8];
+    unpack8(__ldg(xr + v), xf);
+#pragma unroll
+    for (int c = 0; c < kMaxE; ++c) {
+      if (c < r) {
+        float wf[8];
+        unpack8(__ldg(reinterpret_cast<const uint4*>(Wg + (size_t)c * h) + v), wf);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) acc[c] = fmaf(xf[q], wf[q], acc[c]);
+      }
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < kMaxE; ++c) {
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], s);
+    if (lane == 0) s_part[warp][c] = acc[c];
+  }
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+  float l[kMaxE];
+  for (int c = 0; c < r; ++c) {
+    float v = 0.f;
+    for (int w = 0; w < 8; ++w) v += s_part[w][c];
+    l[c] = v;
+  }
+  int sel[kMaxE];
+  float p[kMaxE];
+  unsigned left = (1u << r) - 1u;
+  for (int m = 0; m < k; ++m) {
+    int best = -1;
+    for (int c = 0; c < r; ++c)
+      if (((left >> c) & 1u) && (best < 0 || l[c] > l[best])) best = c;
+    sel[m] = best;
+    left &= ~(1u << best);
+    p[m] = expf(l[best] - l[sel[0]]);
+  }
+  float total = 0.f;
+  for (int m = 0; m < k; ++m) total += p[m];
+  float tail[kMaxE + 1];
+  tail[k] = 0.f;
+  for (int m = k - 1; m >= 1; --m) tail[m] = tail[m + 1] + p[m];
+  int istar = k;
+  for (int i = 1; i <= k; ++i)
+    if (tail[i] <= beta * total) { istar = i; break; }
+  float keep = 0.f;
+  for (int m = 0; m < istar; ++m) keep += p[m];
+  for (int m = 0; m < k; ++m) {
+    const float w = m < istar ? p[m] / keep : 0.f;
+    idx[(size_t)t * k + m] = sel[m];
+    wn[(size_t)t * k + m] = w;
+    if (u_idx) u_idx[(size_t)t * k + m] = kept.id[sel[m]];
+    if (u_wn) u_wn[(size_t)t * k + m] = w;
+  }
+  nact[t] = istar;
+  if (u_nact) u_nact[t] = istar;
+}
+
+// Per block of 64 tokens: active pairs per expert, in the column layout scan_kernel reads
+// (the pairs go to the slot-0 column, the skipped pairs to the last column).
+__global__ void __launch_bounds__(kHistCols < 64 ? 64 : kHistCols)
+count_topk_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ nact, int T, int k,
+                  int32_t* __restrict__ blk_hist) {
+  const int t0 = blockIdx.x * kRouteTokPerBlock;
+  const int col = threadIdx.x;
+  if (col >= kHistCols) return;
+  int n = 0;
+  const int t1 = min(T, t0 + kRouteTokPerBlock);
+  if (col == 2 * kMaxE) {
+    for (int t = t0; t < t1; ++t) n += k - nact[t];
+  } else if ((col & 1) == 0) {
+    const int c = col >> 1;
+    for (int t = t0; t < t1; ++t)
+      for (int m = 0; m < nact[t]; ++m) n += (idx[(size_t)t * k + m] == c);
+  }
+  blk_hist[(size_t)blockIdx.x * kHistCols + col] = n;
+}
+
+// Position of pair (t, m): start of the expert's group + pairs of that expert in earlier
+// blocks + pairs of that expert among the earlier tokens of this block.
+__global__ void __launch_bounds__(kRouteTokPerBlock)
+scatter_topk_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ nact,
+                    const int32_t* __restrict__ blk_base, const Meta* __restrict__ meta, int T,
+                    int k, int32_t* __restrict__ pair_pos, int32_t* __restrict__ row_token) {
+  __shared__ int s_e[kRouteTokPerBlock][kMaxE];
+  const int tl = threadIdx.x;
+  const int t = blockIdx.x * kRouteTokPerBlock + tl;
+  for (int m = 0; m < k; ++m) s_e[tl][m] = (t < T && m < nact[t]) ? idx[(size_t)t * k + m] : -1;
+  __syncthreads();
+  if (t >= T) return;
+  for (int m = 0; m < k; ++m) {
+    const int c = s_e[tl][m];
+    int pos = -1;
+    if (c >= 0) {
+      int rank = 0;
+      for (int i = 0; i < tl; ++i)
+        for (int q = 0; q < k; ++q) rank += (s_e[i][q] == c);
+      pos = meta->off[c] + blk_base[(size_t)blockIdx.x * kMaxE + c] + rank;
+      row_token[pos] = t;
+    }
+    pair_pos[(size_t)t * k + m] = pos;
+  }
+}
+
+__global__ void __launch_bounds__(128)
+combine_topk_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
+                    const int32_t* __restrict__ pair_pos, const float* __restrict__ wn, int k,
+                    int T, int h, bf16* y) {
+  const int t = blockIdx.x;
+  const int nvec = h >> 3;
+  for (int v = blockIdx.y * blockDim.x + threadIdx.x; v < nvec; v += gridDim.y * blockDim.x) {
+    float z[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) z[q] = 0.f;
+    for (int m = 0; m < k; ++m) {
+      const int p = pair_pos[(size_t)t * k + m];
+      if (p < 0) continue;
+      const float w = wn[(size_t)t * k + m];
+      float a[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) a[q] = 0.f;
+      for (int s = 0; s < ksplit; ++s) {
+        const float4* o = reinterpret_cast<const float4*>(O + s * split_stride + (size_t)p * h) + 2 * v;
+        const float4 q0 = o[0], q1 = o[1];
+        a[0] += q0.x; a[1] += q0.y; a[2] += q0.z; a[3] += q0.w;
+        a[4] += q1.x; a[5] += q1.y; a[6] += q1.z; a[7] += q1.w;
+      }
+#pragma unroll
+      for (int q = 0; q < 8; ++q) z[q] = fmaf(w, a[q], z[q]);
+    }
+    uint4 outv;
+    outv.x = pack2(z[0], z[1]); outv.y = pack2(z[2], z[3]);
+    outv.z = pack2(z[4], z[5]); outv.w = pack2(z[6], z[7]);
+    reinterpret_cast<uint4*>(y + (size_t)t * h)[v] = outv;
+  }
+}
+
 // --------------------------------------------------------------------------- co-selection
 
 // counts[a][b] += 1 for every token whose top-2 is (a, b) (App. A.1).  Integer counts: block
@@ -657,6 +816,38 @@ cudaError_t launch_combine(const float* O, int ksplit, size_t split_stride, cons
   if (T > 4096) ychunks = 1;  // plenty of blocks already
   return launch_pdl(combine_kernel, dim3(T, ychunks), dim3(128), 0, st, O, ksplit, split_stride,
                     pair_pos, wn, residual, T, h, y);
+}
+
+cudaError_t launch_router_topk(const bf16* x, const bf16* Wg, int T, int h, int r, int k, float beta,
+                               const KeptIds& kept, int32_t* idx, float* wn, int32_t* nact,
+                               int32_t* u_idx, float* u_wn, int32_t* u_nact, cudaStream_t st) {
+  router_topk_kernel<<<T, 256, 0, st>>>(x, Wg, T, h, r, k, beta, kept, idx, wn, nact, u_idx, u_wn, u_nact);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_count_topk(const int32_t* idx, const int32_t* nact, int T, int k,
+                              int32_t* blk_hist, cudaStream_t st) {
+  const int nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
+  count_topk_kernel<<<nblk, kHistCols < 64 ? 64 : kHistCols, 0, st>>>(idx, nact, T, k, blk_hist);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scatter_topk(const int32_t* idx, const int32_t* nact, const int32_t* blk_base,
+                                const Meta* meta, int T, int k, int32_t* pair_pos,
+                                int32_t* row_token, cudaStream_t st) {
+  const int nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
+  scatter_topk_kernel<<<nblk, kRouteTokPerBlock, 0, st>>>(idx, nact, blk_base, meta, T, k, pair_pos,
+                                                          row_token);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_combine_topk(const float* O, int ksplit, size_t split_stride,
+                                const int32_t* pair_pos, const float* wn, int k, int T, int h,
+                                bf16* y, cudaStream_t st) {
+  int ychunks = ((h >> 3) + 127) / 128;
+  if (T > 4096) ychunks = 1;
+  combine_topk_kernel<<<dim3(T, ychunks), 128, 0, st>>>(O, ksplit, split_stride, pair_pos, wn, k, T, h, y);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_coselection(const int32_t* idx, int T, int E, const KeptIds& kept, int32_t* counts,

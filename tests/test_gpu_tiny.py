@@ -303,3 +303,39 @@ def test_progressive_search_matches_oracle(setup, r):
     fn = float(F_ref.double().norm())
     assert np.abs(np.array(pg) - np.array(lw)).max() <= 2 ** -8 * fn
     layer.close()
+
+
+@pytest.mark.parametrize("E_,kept,k,T,beta", [
+    (16, 0xFFFF, 4, 300, 0.0), (16, 0xFFFF, 4, 300, 0.3), (16, 0xF0F3, 3, 1000, 0.2),
+    (8, 0xFF, 2, 256, 0.3), (8, 0xFF, 1, 64, 0.0), (8, 0b10111101, 6, 40, 0.15), (16, 0xFFFF, 8, 33, 0.4),
+])
+def test_forward_topk_generalised_skipping(E_, kept, k, T, beta):
+    build.build()
+    h, f = 128, 192
+    W = synth.make_layer_weights(h, f, E_, seed=51)
+    b = synth.bf16_bits
+    x = synth.make_tokens(T, h, seed=52)
+    ora = O.moe_forward_topk(b(x), b(W.W_gate), b(W.W1), b(W.W3), b(W.W2), kept, k, beta)
+    layer = binding.MoeLayer(W.W_gate.to(DEV), W.W1.to(DEV), W.W3.to(DEV), W.W2.to(DEV), kept)
+    y, idx, wn, na = layer.forward_topk(x.to(DEV), k, beta, record=True)
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+    idx, wn, na = idx.cpu().numpy(), wn.cpu().numpy(), na.cpu().numpy()
+    # near-ties: an adjacent gap below 1e-3 among the k+1 largest kept logits
+    keptv = np.array([(kept >> e) & 1 for e in range(E_)], bool)
+    srt = -np.sort(-np.where(keptv[None, :], ora["logits"].astype(np.float64), -np.inf), axis=1)
+    tie = (np.diff(-srt[:, :min(k + 1, int(keptv.sum()))], axis=1) < P.LOGIT_GAP_TOL).any(1)
+    assert tie.mean() < 0.1
+    assert np.array_equal(idx[~tie], ora["idx"][~tie])
+    same_idx = (idx == ora["idx"]).all(1)
+    # the decision i* may differ only where a tail mass sits on the threshold
+    sel = np.take_along_axis(ora["logits"].astype(np.float64), ora["idx"].astype(np.int64), 1)
+    p = np.exp(sel - sel[:, :1])
+    fr = np.stack([p[:, i:].sum(1) for i in range(1, k + 1)], 1) / p.sum(1, keepdims=True)
+    close = (np.abs(fr - beta) < P.RATIO_TOL).any(1)
+    chk = same_idx & ~close
+    assert np.array_equal(na[chk], ora["n_active"][chk])
+    both = same_idx & (na == ora["n_active"])
+    np.testing.assert_allclose(wn[both], ora["wn"][both], rtol=2e-5, atol=1e-7)
+    P.check_outputs(b(y), ora["y"], both)
+    layer.close()
