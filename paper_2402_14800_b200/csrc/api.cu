@@ -63,7 +63,7 @@ struct Workspace {
   Buf row_token, xperm, act, O, tail;
   CUtensorMap tok_x[4], tok_act[4];  // boxes of 16/32/64/128 rows over xperm and act
   // search scratch
-  Buf s_logits, s_yall, s_act, s_subsets, s_partial, s_loss_sq, s_losses, s_xpad, s_meta;
+  Buf s_logits, s_yall, s_act, s_subsets, s_partial, s_loss_sq, s_losses, s_xpad, s_meta, s_xperm, s_rowtok;
   // host staging and stack scratch
   Buf hx, hy, xn, cosel;
   // general top-k path
@@ -88,6 +88,7 @@ struct moe_layer {
   size_t weight_bytes = 0;
   cudaStream_t stream = 0;
   bool debug_simt = false;
+  bool search_dense = false;  // MOE_SEARCH_DENSE=1: evaluate all E experts per token in the search
   CUtensorMap w13_256, w13_128, w2_256, w2_128;
   Workspace own;
   Workspace* ws = &own;
@@ -378,6 +379,8 @@ moe_layer_t* moe_layer_create(const void* W_gate, const void* W1, const void* W3
   for (int c = L->r; c < kMaxE; ++c) L->kept.id[c] = 0;
   const char* dbg = getenv("MOE_DEBUG_SIMT");
   L->debug_simt = dbg && dbg[0] == '1';
+  const char* dense = getenv("MOE_SEARCH_DENSE");
+  L->search_dense = dense && dense[0] == '1';
 
   const size_t n_gate = (size_t)L->r * h * 2, n_13 = (size_t)L->r * 2 * f * h * 2,
                n_2 = (size_t)L->r * h * f * 2;
@@ -430,7 +433,7 @@ void moe_layer_destroy(moe_layer_t* L) {
   Buf* bufs[] = {&L->own.idx, &L->own.wn, &L->own.ratio, &L->own.skipped, &L->own.blk_hist, &L->own.blk_base, &L->own.pair_pos,
                  &L->own.meta, &L->own.status, &L->own.sel, &L->own.row_token, &L->own.xperm, &L->own.act, &L->own.O, &L->own.tail,
                  &L->own.s_logits, &L->own.s_yall, &L->own.s_act, &L->own.s_subsets, &L->own.s_partial, &L->own.s_loss_sq,
-                 &L->own.s_losses, &L->own.s_xpad, &L->own.s_meta, &L->own.hx, &L->own.hy, &L->own.xn, &L->own.cosel, &L->own.k_idx, &L->own.k_wn, &L->own.k_pos, &L->own.k_nact};
+                 &L->own.s_losses, &L->own.s_xpad, &L->own.s_meta, &L->own.s_xperm, &L->own.s_rowtok, &L->own.hx, &L->own.hy, &L->own.xn, &L->own.cosel, &L->own.k_idx, &L->own.k_wn, &L->own.k_pos, &L->own.k_nact};
   for (Buf* b : bufs) release(L, *b);
   for (cudaEvent_t e : L->prof_ev) cudaEventDestroy(e);
   if (L->Wg) cudaFree(L->Wg);
@@ -482,7 +485,7 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
   int32_t* idx = (int32_t*)W.k_idx.p;
   int32_t* nact = (int32_t*)W.k_nact.p;
   CUDA_TRY(launch_router_topk((const bf16*)x, L->Wg, T, L->h, L->r, k, beta, L->kept, idx,
-                              (float*)W.k_wn.p, nact, idx_out, wn_out, n_active_out, st));
+                              (float*)W.k_wn.p, nact, idx_out, wn_out, n_active_out, nullptr, st));
   CUDA_TRY(launch_count_topk(idx, nact, T, k, (int32_t*)W.blk_hist.p, st));
   CUDA_TRY(launch_scan((int32_t*)W.blk_hist.p, nblk, L->r, dec ? 16 : kTileRows, (int32_t*)W.blk_base.p,
                        meta, nullptr, nullptr, nullptr, L->kept, L->E, st));
@@ -626,63 +629,125 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
     }
   }
 
-  const int Tc = T < 8192 ? T : 8192;                     // tokens per all-experts chunk
+  const int Tc = T < 8192 ? T : 8192;  // tokens per chunk of expert evaluations
   const int Tc_pad = (int)align_up((size_t)Tc, kTileRows);
+  const int nchunks = (T + Tc - 1) / Tc;
   const int nblk_enum = enumerate_num_blocks(T, (int)nC);
-  if ((rc = grow(L, L->ws->s_logits, (size_t)T * E * 4))) return rc;
-  if ((rc = grow(L, L->ws->s_yall, (size_t)T * E * h * 2))) return rc;
-  if ((rc = grow(L, L->ws->s_act, ((size_t)E * Tc_pad + kTileRows) * f * 2))) return rc;
-  if ((rc = grow(L, L->ws->s_subsets, (size_t)nC * 4))) return rc;
-  if ((rc = grow(L, L->ws->s_partial, (size_t)nblk_enum * nC * 4))) return rc;
-  if ((rc = grow(L, L->ws->s_loss_sq, (size_t)nC * 8))) return rc;
-  if ((rc = grow(L, L->ws->s_losses, (size_t)nC * 4))) return rc;
-  if ((rc = grow(L, L->ws->s_meta, sizeof(Meta)))) return rc;
-  CUDA_TRY(cudaMemcpyAsync(L->ws->s_subsets.p, masks.data(), (size_t)nC * 4, cudaMemcpyHostToDevice, st));
-
-  // token-side operand of the gate/up GEMM: x itself (padded copy when shorter than one box)
-  const bf16* xa = (const bf16*)x_calib;
-  uint64_t xa_rows = (uint64_t)T;
-  if (T < kTileRows) {
-    if ((rc = grow(L, L->ws->s_xpad, (size_t)kTileRows * h * 2))) return rc;
-    CUDA_TRY(cudaMemsetAsync(L->ws->s_xpad.p, 0, (size_t)kTileRows * h * 2, st));
-    CUDA_TRY(cudaMemcpyAsync(L->ws->s_xpad.p, x_calib, (size_t)T * h * 2, cudaMemcpyDeviceToDevice, st));
-    xa = (const bf16*)L->ws->s_xpad.p;
-    xa_rows = kTileRows;
-  }
+  // A subset of r experts always contains two of a token's K = E - r + 2 top-ranked experts,
+  // so only those K need to be evaluated per token (all of them when K = E).
+  const int K = E - r + 2;
+  const bool pruned_work = K < E && !L->search_dense;
+  Workspace& W = *L->ws;
+  if ((rc = grow(L, W.s_logits, (size_t)T * E * 4))) return rc;
+  if ((rc = grow(L, W.s_subsets, (size_t)nC * 4))) return rc;
+  if ((rc = grow(L, W.s_partial, (size_t)nblk_enum * nC * 4))) return rc;
+  if ((rc = grow(L, W.s_loss_sq, (size_t)nC * 8))) return rc;
+  if ((rc = grow(L, W.s_losses, (size_t)nC * 4))) return rc;
+  if ((rc = grow(L, W.s_meta, sizeof(Meta)))) return rc;
+  CUDA_TRY(cudaMemcpyAsync(W.s_subsets.p, masks.data(), (size_t)nC * 4, cudaMemcpyHostToDevice, st));
+  Meta* meta = (Meta*)W.s_meta.p;
+  const bool prof_saved = L->prof;
+  L->prof = false;  // stage marks describe moe_forward only
+  EnumSource src = {nullptr, nullptr, 0, 0};
   GemmMaps m_gu, m_dn;
   m_gu.w = L->w13_256;
   m_dn.w = L->w2_256;
-  if ((rc = build_token_maps(m_gu, xa, h, xa_rows))) return rc;
-  if ((rc = build_token_maps(m_dn, L->ws->s_act.p, f, (uint64_t)E * Tc_pad + kTileRows))) return rc;
 
-  // all logits (Sec. 3.2: the unpruned layer's routing), then every expert on every token
-  RouteOut ro;
-  memset(&ro, 0, sizeof(ro));
-  ro.idx = (int32_t*)L->ws->idx.p; ro.wn = (float*)L->ws->wn.p; ro.ratio = (float*)L->ws->ratio.p;
-  ro.skipped = (uint8_t*)L->ws->skipped.p; ro.logits = (float*)L->ws->s_logits.p;
-  CUDA_TRY(launch_router((const bf16*)x_calib, L->Wg, T, h, E, 0.f, L->kept, ro, st));
-  Meta* meta = (Meta*)L->ws->s_meta.p;
-  const bool prof_saved = L->prof;
-  L->prof = false;  // stage marks describe moe_forward only
-  for (int t0 = 0; t0 < T; t0 += Tc) {
-    const int rows = (T - t0) < Tc ? (T - t0) : Tc;
-    CUDA_TRY(launch_set_dense_meta(meta, E, rows, Tc_pad, st));
-    GemmArgs gu, dn;
-    memset(&gu, 0, sizeof(gu));
-    memset(&dn, 0, sizeof(dn));
-    gu.a_row_base = t0; gu.a_off_mul = 0; gu.out_off_mul = 1; gu.out_ld = f; gu.out = L->ws->s_act.p;
-    dn.a_off_mul = 1; dn.out_row_base = t0; dn.out_off_mul = 0; dn.out_col_mul = h;
-    dn.out_ld = (long long)E * h; dn.out = L->ws->s_yall.p;
-    if ((rc = run_expert_gemms(L, meta, false, m_gu, m_dn, gu, dn, kOutBf16, xa,
-                               (const bf16*)L->ws->s_act.p, rows))) {
-      L->prof = prof_saved;
-      return rc;
+  if (pruned_work) {
+    const int rows_chunk = (int)align_up((size_t)K * Tc + (size_t)E * kTileRows, kTileRows);
+    if ((rc = grow(L, W.s_yall, (size_t)nchunks * rows_chunk * h * 2))) return rc;
+    if ((rc = grow(L, W.s_act, ((size_t)rows_chunk + kTileRows) * f * 2))) return rc;
+    if ((rc = grow(L, W.s_xperm, ((size_t)rows_chunk + kTileRows) * h * 2))) return rc;
+    if ((rc = grow(L, W.s_rowtok, (size_t)rows_chunk * 4))) return rc;
+    if ((rc = grow(L, W.k_idx, (size_t)T * K * 4))) return rc;
+    if ((rc = grow(L, W.k_wn, (size_t)T * K * 4))) return rc;
+    if ((rc = grow(L, W.k_pos, (size_t)T * K * 4))) return rc;
+    if ((rc = grow(L, W.k_nact, (size_t)T * 4))) return rc;
+    if ((rc = build_token_maps(m_gu, W.s_xperm.p, h, (uint64_t)rows_chunk + kTileRows))) return rc;
+    if ((rc = build_token_maps(m_dn, W.s_act.p, f, (uint64_t)rows_chunk + kTileRows))) return rc;
+    for (int c = 0; c < nchunks; ++c) {
+      const int t0 = c * Tc;
+      const int rows = (T - t0) < Tc ? (T - t0) : Tc;
+      const int nblk = (rows + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
+      const bf16* xc = (const bf16*)x_calib + (size_t)t0 * h;
+      int32_t* idx = (int32_t*)W.k_idx.p + (size_t)t0 * K;
+      int32_t* nact = (int32_t*)W.k_nact.p + t0;
+      int32_t* pos = (int32_t*)W.k_pos.p + (size_t)t0 * K;
+      // beta = -1: the skipping rule never fires, every token keeps its K top-ranked experts
+      cudaError_t e = launch_router_topk(xc, L->Wg, rows, h, E, K, -1.0f, L->kept, idx,
+                                         (float*)W.k_wn.p + (size_t)t0 * K, nact, nullptr, nullptr,
+                                         nullptr, (float*)W.s_logits.p + (size_t)t0 * E, st);
+      if (e == cudaSuccess) e = launch_count_topk(idx, nact, rows, K, (int32_t*)W.blk_hist.p, st);
+      if (e == cudaSuccess)
+        e = launch_scan((int32_t*)W.blk_hist.p, nblk, E, kTileRows, (int32_t*)W.blk_base.p, meta, nullptr,
+                        nullptr, nullptr, L->kept, E, st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(W.s_rowtok.p, 0xff, (size_t)rows_chunk * 4, st);
+      if (e == cudaSuccess)
+        e = launch_scatter_topk(idx, nact, (int32_t*)W.blk_base.p, meta, rows, K, pos,
+                                (int32_t*)W.s_rowtok.p, st);
+      if (e == cudaSuccess)
+        e = launch_gather(xc, (int32_t*)W.s_rowtok.p, meta, h, rows_chunk, (bf16*)W.s_xperm.p, st);
+      if (e != cudaSuccess) {
+        L->prof = prof_saved;
+        return fail(MOE_ERR_CUDA, "search permutation: %s", cudaGetErrorString(e));
+      }
+      GemmArgs gu, dn;
+      memset(&gu, 0, sizeof(gu));
+      memset(&dn, 0, sizeof(dn));
+      gu.a_off_mul = 1; gu.out_off_mul = 1; gu.out_ld = f; gu.out = W.s_act.p;
+      dn.a_off_mul = 1; dn.out_off_mul = 1; dn.out_row_base = c * rows_chunk; dn.out_ld = h;
+      dn.out = W.s_yall.p;
+      if ((rc = run_expert_gemms(L, meta, false, m_gu, m_dn, gu, dn, kOutBf16, (const bf16*)W.s_xperm.p,
+                                 (const bf16*)W.s_act.p, rows_chunk))) {
+        L->prof = prof_saved;
+        return rc;
+      }
+    }
+    src.topk_idx = (const int32_t*)W.k_idx.p;
+    src.pair_pos = (const int32_t*)W.k_pos.p;
+    src.chunk_tokens = Tc;
+    src.chunk_rows = rows_chunk;
+  } else {
+    if ((rc = grow(L, W.s_yall, (size_t)T * E * h * 2))) return rc;
+    if ((rc = grow(L, W.s_act, ((size_t)E * Tc_pad + kTileRows) * f * 2))) return rc;
+    // token-side operand of the gate/up GEMM: x itself (padded copy when shorter than one box)
+    const bf16* xa = (const bf16*)x_calib;
+    uint64_t xa_rows = (uint64_t)T;
+    if (T < kTileRows) {
+      if ((rc = grow(L, W.s_xpad, (size_t)kTileRows * h * 2))) return rc;
+      CUDA_TRY(cudaMemsetAsync(W.s_xpad.p, 0, (size_t)kTileRows * h * 2, st));
+      CUDA_TRY(cudaMemcpyAsync(W.s_xpad.p, x_calib, (size_t)T * h * 2, cudaMemcpyDeviceToDevice, st));
+      xa = (const bf16*)W.s_xpad.p;
+      xa_rows = kTileRows;
+    }
+    if ((rc = build_token_maps(m_gu, xa, h, xa_rows))) return rc;
+    if ((rc = build_token_maps(m_dn, W.s_act.p, f, (uint64_t)E * Tc_pad + kTileRows))) return rc;
+    // all logits (Sec. 3.2: the unpruned layer's routing), then every expert on every token
+    RouteOut ro;
+    memset(&ro, 0, sizeof(ro));
+    ro.idx = (int32_t*)W.idx.p; ro.wn = (float*)W.wn.p; ro.ratio = (float*)W.ratio.p;
+    ro.skipped = (uint8_t*)W.skipped.p; ro.logits = (float*)W.s_logits.p;
+    CUDA_TRY(launch_router((const bf16*)x_calib, L->Wg, T, h, E, 0.f, L->kept, ro, st));
+    for (int t0 = 0; t0 < T; t0 += Tc) {
+      const int rows = (T - t0) < Tc ? (T - t0) : Tc;
+      CUDA_TRY(launch_set_dense_meta(meta, E, rows, Tc_pad, st));
+      GemmArgs gu, dn;
+      memset(&gu, 0, sizeof(gu));
+      memset(&dn, 0, sizeof(dn));
+      gu.a_row_base = t0; gu.a_off_mul = 0; gu.out_off_mul = 1; gu.out_ld = f; gu.out = W.s_act.p;
+      dn.a_off_mul = 1; dn.out_row_base = t0; dn.out_off_mul = 0; dn.out_col_mul = h;
+      dn.out_ld = (long long)E * h; dn.out = W.s_yall.p;
+      if ((rc = run_expert_gemms(L, meta, false, m_gu, m_dn, gu, dn, kOutBf16, xa,
+                                 (const bf16*)W.s_act.p, rows))) {
+        L->prof = prof_saved;
+        return rc;
+      }
     }
   }
   L->prof = prof_saved;
-  CUDA_TRY(launch_enumerate((const float*)L->ws->s_logits.p, (const bf16*)L->ws->s_yall.p, T, E, r, h,
-                            (const uint32_t*)L->ws->s_subsets.p, (int)nC, (float*)L->ws->s_partial.p,
-                            (double*)L->ws->s_loss_sq.p, (float*)L->ws->s_losses.p, F_ref, st));
+  CUDA_TRY(launch_enumerate((const float*)W.s_logits.p, (const bf16*)W.s_yall.p, T, E, r, h,
+                            (const uint32_t*)W.s_subsets.p, (int)nC, (float*)W.s_partial.p,
+                            (double*)W.s_loss_sq.p, (float*)W.s_losses.p, F_ref, src, st));
   CUDA_TRY(cudaMemcpyAsync(losses, L->ws->s_losses.p, (size_t)nC * 4, cudaMemcpyDeviceToHost, st));
   if ((rc = check_status(L))) return rc;
   long best = 0;

@@ -106,7 +106,8 @@ cudaError_t launch_combine(const float* O, int ksplit, size_t split_stride, cons
 // general top-k path (k slots per token instead of two)
 cudaError_t launch_router_topk(const bf16* x, const bf16* Wg, int T, int h, int r, int k, float beta,
                                const KeptIds& kept, int32_t* idx, float* wn, int32_t* nact,
-                               int32_t* u_idx, float* u_wn, int32_t* u_nact, cudaStream_t st);
+                               int32_t* u_idx, float* u_wn, int32_t* u_nact, float* logits,
+                               cudaStream_t st);
 cudaError_t launch_count_topk(const int32_t* idx, const int32_t* nact, int T, int k,
                               int32_t* blk_hist, cudaStream_t st);
 cudaError_t launch_scatter_topk(const int32_t* idx, const int32_t* nact, const int32_t* blk_base,
@@ -173,9 +174,20 @@ cudaError_t launch_simt_down(const bf16* A, const bf16* W2, const GemmArgs& a, i
 cudaError_t gemm_set_attributes();
 
 // ---- search (search.cu) ---------------------------------------------------------------
+// Where the enumeration finds the expert outputs.  Dense (topk_idx == null): Yall[T][E][h].
+// Pruned work: only each token's K = E - r + 2 top-ranked experts were evaluated;
+// topk_idx[T][K] lists them in rank order and their outputs are rows of a permuted buffer,
+// row (t / chunk_tokens) * chunk_rows + pair_pos[t][rank].
+struct EnumSource {
+  const int32_t* topk_idx;
+  const int32_t* pair_pos;
+  int chunk_tokens;
+  int chunk_rows;
+};
 int enumerate_num_blocks(int T, int nC);
 cudaError_t launch_enumerate(const float* logits, const bf16* Yall, int T, int E, int r, int h,
                              const uint32_t* subsets, int nC, float* partial, double* loss_sq,
-                             float* losses, const float* Fref, cudaStream_t st);
+                             float* losses, const float* Fref, const EnumSource& src,
+                             cudaStream_t st);
 
 }  // namespace moe

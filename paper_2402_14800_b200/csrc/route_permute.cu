@@ -458,7 +458,7 @@ __global__ void __launch_bounds__(256)
 router_topk_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, int h, int r,
                    int k, float beta, KeptIds kept, int32_t* __restrict__ idx,
                    float* __restrict__ wn, int32_t* __restrict__ nact, int32_t* u_idx, float* u_wn,
-                   int32_t* u_nact) {
+                   int32_t* u_nact, float* logits) {
   __shared__ float s_part[8][kMaxE];
   const int t = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -493,6 +493,7 @@ router_topk_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int 
     float v = 0.f;
     for (int w = 0; w < 8; ++w) v += s_part[w][c];
     l[c] = v;
+    if (logits) logits[(size_t)t * r + c] = v;
   }
   int sel[kMaxE];
   float p[kMaxE];
@@ -820,8 +821,10 @@ cudaError_t launch_combine(const float* O, int ksplit, size_t split_stride, cons
 
 cudaError_t launch_router_topk(const bf16* x, const bf16* Wg, int T, int h, int r, int k, float beta,
                                const KeptIds& kept, int32_t* idx, float* wn, int32_t* nact,
-                               int32_t* u_idx, float* u_wn, int32_t* u_nact, cudaStream_t st) {
-  router_topk_kernel<<<T, 256, 0, st>>>(x, Wg, T, h, r, k, beta, kept, idx, wn, nact, u_idx, u_wn, u_nact);
+                               int32_t* u_idx, float* u_wn, int32_t* u_nact, float* logits,
+                               cudaStream_t st) {
+  router_topk_kernel<<<T, 256, 0, st>>>(x, Wg, T, h, r, k, beta, kept, idx, wn, nact, u_idx, u_wn, u_nact,
+                                        logits);
   return cudaGetLastError();
 }
 

@@ -38,7 +38,8 @@ __device__ __forceinline__ void pair_weights(float l_first, float l_second, floa
 // unpruned output built from the two top-ranked experts.
 template <int K>
 __device__ __forceinline__ void pair_errors_fast(const bf16* __restrict__ Yt, int h,
-                                                 const int* order, const float* l, int lane,
+                                                 const int* order, const int* rowoff,
+                                                 const float* l, int lane,
                                                  float* s_err /* [16*16] */,
                                                  const float* __restrict__ ref) {
   constexpr int NP = K * (K - 1) / 2;
@@ -55,7 +56,7 @@ __device__ __forceinline__ void pair_errors_fast(const bf16* __restrict__ Yt, in
   }
   const uint4* rows[K];
 #pragma unroll
-  for (int i = 0; i < K; ++i) rows[i] = reinterpret_cast<const uint4*>(Yt + (size_t)order[i] * h);
+  for (int i = 0; i < K; ++i) rows[i] = reinterpret_cast<const uint4*>(Yt + (size_t)rowoff[i] * h);
   for (int v = lane; v < (h >> 3); v += 32) {
     float y[K][8];
 #pragma unroll
@@ -94,18 +95,19 @@ __device__ __forceinline__ void pair_errors_fast(const bf16* __restrict__ Yt, in
 
 // The same for any K, one pair at a time (rows are re-read from cache).
 __device__ __forceinline__ void pair_errors_generic(const bf16* __restrict__ Yt, int h, int K,
-                                                    const int* order, const float* l, int lane,
-                                                    float* s_err, const float* __restrict__ ref) {
+                                                    const int* order, const int* rowoff,
+                                                    const float* l, int lane, float* s_err,
+                                                    const float* __restrict__ ref) {
   float w0, w1;
   pair_weights(l[order[0]], l[order[1]], w0, w1);
-  const uint4* r0 = reinterpret_cast<const uint4*>(Yt + (size_t)order[0] * h);
-  const uint4* r1 = reinterpret_cast<const uint4*>(Yt + (size_t)order[1] * h);
+  const uint4* r0 = reinterpret_cast<const uint4*>(Yt + (size_t)rowoff[0] * h);
+  const uint4* r1 = reinterpret_cast<const uint4*>(Yt + (size_t)rowoff[1] * h);
   for (int i = 0; i < K; ++i)
     for (int j = i + 1; j < K; ++j) {
       float wa, wb;
       pair_weights(l[order[i]], l[order[j]], wa, wb);
-      const uint4* ri = reinterpret_cast<const uint4*>(Yt + (size_t)order[i] * h);
-      const uint4* rj = reinterpret_cast<const uint4*>(Yt + (size_t)order[j] * h);
+      const uint4* ri = reinterpret_cast<const uint4*>(Yt + (size_t)rowoff[i] * h);
+      const uint4* rj = reinterpret_cast<const uint4*>(Yt + (size_t)rowoff[j] * h);
       float e = 0.f;
       for (int v = lane; v < (h >> 3); v += 32) {
         float y0[8], y1[8], yi[8], yj[8];
@@ -129,7 +131,7 @@ __device__ __forceinline__ void pair_errors_generic(const bf16* __restrict__ Yt,
 __global__ void __launch_bounds__(128)
 enumerate_kernel(const float* __restrict__ logits, const bf16* __restrict__ Yall, int T, int E,
                  int r, int h, const uint32_t* __restrict__ subsets, int nC,
-                 float* __restrict__ partial, const float* __restrict__ Fref) {
+                 float* __restrict__ partial, const float* __restrict__ Fref, EnumSource src) {
   extern __shared__ float s_dyn[];
   const int nwarps = blockDim.x >> 5;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -139,6 +141,7 @@ enumerate_kernel(const float* __restrict__ logits, const bf16* __restrict__ Yall
   int* base_order = reinterpret_cast<int*>(base_err + nwarps * (kMaxE * kMaxE));
   int* s_order = base_order + warp * kMaxE;
   float* s_l = reinterpret_cast<float*>(base_order + nwarps * kMaxE) + warp * kMaxE;
+  int* s_row = reinterpret_cast<int*>(base_order + 2 * nwarps * kMaxE) + warp * kMaxE;
 
   for (int s = lane; s < nC; s += 32) acc[s] = 0.f;
   const int K = E - r + 2;
@@ -153,30 +156,38 @@ enumerate_kernel(const float* __restrict__ logits, const bf16* __restrict__ Yall
       s_l[lane] = mine;
     }
     __syncwarp();
-    if (lane < E) {
+    if (src.topk_idx) {
+      // only the K top-ranked experts were evaluated; they are listed in rank order, and their
+      // outputs sit in the permuted row pair_pos[t][rank] of the token's chunk
+      if (lane < K) {
+        s_order[lane] = src.topk_idx[(size_t)t * K + lane];
+        s_row[lane] = (t / src.chunk_tokens) * src.chunk_rows + src.pair_pos[(size_t)t * K + lane];
+      }
+    } else if (lane < E) {
       int rank = 0;
       for (int e = 0; e < E; ++e) {
         const float o = s_l[e];
         rank += (o > mine) || (o == mine && e < lane);
       }
       s_order[rank] = lane;
+      s_row[rank] = lane;
     }
     __syncwarp();
-    const bf16* Yt = Yall + (size_t)t * E * h;
+    const bf16* Yt = src.topk_idx ? Yall : Yall + (size_t)t * E * h;
     const float* ref = Fref ? Fref + (size_t)t * h : nullptr;
     switch (K) {
-      case 2: pair_errors_fast<2>(Yt, h, s_order, s_l, lane, s_err, ref); break;
-      case 3: pair_errors_fast<3>(Yt, h, s_order, s_l, lane, s_err, ref); break;
-      case 4: pair_errors_fast<4>(Yt, h, s_order, s_l, lane, s_err, ref); break;
-      case 5: pair_errors_fast<5>(Yt, h, s_order, s_l, lane, s_err, ref); break;
-      case 6: pair_errors_fast<6>(Yt, h, s_order, s_l, lane, s_err, ref); break;
-      default: pair_errors_generic(Yt, h, K, s_order, s_l, lane, s_err, ref); break;
+      case 2: pair_errors_fast<2>(Yt, h, s_order, s_row, s_l, lane, s_err, ref); break;
+      case 3: pair_errors_fast<3>(Yt, h, s_order, s_row, s_l, lane, s_err, ref); break;
+      case 4: pair_errors_fast<4>(Yt, h, s_order, s_row, s_l, lane, s_err, ref); break;
+      case 5: pair_errors_fast<5>(Yt, h, s_order, s_row, s_l, lane, s_err, ref); break;
+      case 6: pair_errors_fast<6>(Yt, h, s_order, s_row, s_l, lane, s_err, ref); break;
+      default: pair_errors_generic(Yt, h, K, s_order, s_row, s_l, lane, s_err, ref); break;
     }
     __syncwarp();
     for (int s = lane; s < nC; s += 32) {
       const uint32_t mask = subsets[s];
       int i = -1, j = -1;
-      for (int q = 0; q < E; ++q) {
+      for (int q = 0; q < K; ++q) {  // the two best kept experts are always among the top K
         if ((mask >> s_order[q]) & 1u) {
           if (i < 0) i = q;
           else { j = q; break; }
@@ -217,10 +228,11 @@ int enumerate_num_blocks(int T, int nC) {
 
 cudaError_t launch_enumerate(const float* logits, const bf16* Yall, int T, int E, int r, int h,
                              const uint32_t* subsets, int nC, float* partial, double* loss_sq,
-                             float* losses, const float* Fref, cudaStream_t st) {
+                             float* losses, const float* Fref, const EnumSource& src,
+                             cudaStream_t st) {
   const int nw = warps_for(nC);
   const int nblk = enumerate_num_blocks(T, nC);
-  const size_t smem = ((size_t)nw * nC + (size_t)nw * kMaxE * kMaxE + 2 * (size_t)nw * kMaxE) * 4;
+  const size_t smem = ((size_t)nw * nC + (size_t)nw * kMaxE * kMaxE + 3 * (size_t)nw * kMaxE) * 4;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(enumerate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -229,7 +241,7 @@ cudaError_t launch_enumerate(const float* logits, const bf16* Yall, int T, int E
     attr_set = true;
   }
   if (smem > 96 * 1024) return cudaErrorInvalidValue;
-  enumerate_kernel<<<nblk, nw * 32, smem, st>>>(logits, Yall, T, E, r, h, subsets, nC, partial, Fref);
+  enumerate_kernel<<<nblk, nw * 32, smem, st>>>(logits, Yall, T, E, r, h, subsets, nC, partial, Fref, src);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   reduce_partials_kernel<<<(nC + 127) / 128, 128, 0, st>>>(partial, nblk, nC, loss_sq, losses);
