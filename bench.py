@@ -391,9 +391,11 @@ def run_ours(a):
                                         "frac": dn_flop / (dn_ms * 1e-3) / 1e12 / peaks["tf_sust"]},
                         "whole_step_frac": (gu_flop + dn_flop) / (ms_step * 1e-3) / 1e12 / peaks["tf_sust"]}
     elif a.workload == "search":
-        flop = 98 * 0 + 2 * (6 * T * E * H * F)  # two searches, each one all-experts GEMM pass
+        # two searches (r = 6, r = 4); each evaluates a token's E - r + 2 top-ranked experts
+        dense = os.environ.get("MOE_SEARCH_DENSE", "") == "1"
+        flop = sum(6 * T * (E if dense else E - r_ + 2) * H * F for r_ in (6, 4))
         ach = flop / (ms_step * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel (all experts, whole search step)",
+        roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel (expert evaluations of the search, whole step)",
                     "achieved": ach, "peak": peaks["tf_sust"], "unit": "TFLOP/s",
                     "frac": ach / peaks["tf_sust"], "traffic": None,
                     "peak_source": peaks["source"] + " (sustained bf16)"}
@@ -432,7 +434,7 @@ def run_ours(a):
         gpu_launches = launches_per_step * a.steps if launches_per_step else None
         if a.workload == "search":
             chunks = (T + 8191) // 8192
-            gpu_launches = a.steps * 2 * (1 + chunks * 3 + 2)
+            gpu_launches = a.steps * 2 * (chunks * 7 + 2)  # per chunk: route, count, scan, scatter, gather, 2 GEMMs
         line = {
             "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": a.steps,
             "warmup": max(a.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,

@@ -164,7 +164,7 @@ cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps&
                                  const GemmArgs& a, cudaStream_t st);
 // Weight rows are the 128-row MMA operand, tokens the narrow one (small T): weights stream once.
 cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
-                                  int kb_per_item, cudaStream_t st);
+                                  int kb_per_item, int max_tokens_per_tile, cudaStream_t st);
 // Plain CUDA-core kernels of the same contractions, for bring-up and debugging only
 // (MOE_DEBUG_SIMT=1); never selected otherwise.
 cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,

@@ -695,32 +695,32 @@ tail_fixup_kernel(const GemmArgs args, int kb_per_item, int gemm_grid) {
   }
   decode_item_w(s_meta, args, sched, sched.full + (int)blockIdx.x * sched.KSt, w);
   const float* slot0 = args.tail + (size_t)(blockIdx.x * sched.KSt) * kTailSlotFloats;
+  // blockIdx.y walks the tokens of the tile (two per block for gate/up, one for down), so each
+  // thread produces one output from nslice independent loads
   if (GATE_UP) {
     // 64 features per tile: rows 32q + s are gate, 32q + 16 + s up
-    for (int idx = threadIdx.x; idx < w.cnt * 64; idx += blockDim.x) {
-      const int n = idx >> 6, fj = idx & 63;
-      const int q = fj >> 4, sft = fj & 15;
-      if (w.mt * 128 + 32 * q >= args.n_w_rows) continue;
-      float g = 0.f, u = 0.f;
-      for (int sub = 0; sub < nslice; ++sub) {
-        const float* t = slot0 + (size_t)sub * kTailSlotFloats + n * 128;
-        g += t[32 * q + sft];
-        u += t[32 * q + 16 + sft];
-      }
-      const int feat = (w.mt * 4 + q) * kInterleave + sft;
-      reinterpret_cast<bf16*>(args.out)[(long long)(w.out_row + n) * args.out_ld + feat] =
-          __float2bfloat16_rn(silu_mul(g, u));
+    const int n = 2 * blockIdx.y + (threadIdx.x >> 6), fj = threadIdx.x & 63;
+    const int q = fj >> 4, sft = fj & 15;
+    if (n >= w.cnt || w.mt * 128 + 32 * q >= args.n_w_rows) return;
+    float g = 0.f, u = 0.f;
+#pragma unroll 4
+    for (int sub = 0; sub < nslice; ++sub) {
+      const float* t = slot0 + (size_t)sub * kTailSlotFloats + n * 128;
+      g += t[32 * q + sft];
+      u += t[32 * q + 16 + sft];
     }
+    const int feat = (w.mt * 4 + q) * kInterleave + sft;
+    reinterpret_cast<bf16*>(args.out)[(long long)(w.out_row + n) * args.out_ld + feat] =
+        __float2bfloat16_rn(silu_mul(g, u));
   } else {
-    for (int idx = threadIdx.x; idx < w.cnt * 128; idx += blockDim.x) {
-      const int n = idx >> 7, col = idx & 127;
-      const int wrow = w.mt * 128 + col;
-      if (wrow >= args.n_w_rows) continue;
-      float v = 0.f;
-      for (int sub = 0; sub < nslice; ++sub) v += slot0[(size_t)sub * kTailSlotFloats + n * 128 + col];
-      reinterpret_cast<float*>(args.out)[(long long)w.ks * args.split_stride +
-                                         (long long)(w.out_row + n) * args.out_ld + wrow] = v;
-    }
+    const int n = blockIdx.y, col = threadIdx.x;
+    const int wrow = w.mt * 128 + col;
+    if (n >= w.cnt || wrow >= args.n_w_rows) return;
+    float v = 0.f;
+#pragma unroll 4
+    for (int sub = 0; sub < nslice; ++sub) v += slot0[(size_t)sub * kTailSlotFloats + n * 128 + col];
+    reinterpret_cast<float*>(args.out)[(long long)w.ks * args.split_stride +
+                                       (long long)(w.out_row + n) * args.out_ld + wrow] = v;
   }
 }
 
@@ -857,18 +857,19 @@ cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps&
 }
 
 cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
-                                  int kb_per_item, cudaStream_t st) {
+                                  int kb_per_item, int max_tokens_per_tile, cudaStream_t st) {
+  const int mt = max_tokens_per_tile < 1 ? 1 : (max_tokens_per_tile > WM_BN ? WM_BN : max_tokens_per_tile);
   const int grid = g_num_sms > 0 ? g_num_sms : 148;
   if (gate_up) {
     cudaError_t e = launch_pdl(gemm_weights_m_kernel<true>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
                                kb_per_item);
     if (e != cudaSuccess || !a.tail) return e;
-    return launch_pdl(tail_fixup_kernel<true>, dim3(grid / 2), dim3(128), 0, st, a, kb_per_item, grid);
+    return launch_pdl(tail_fixup_kernel<true>, dim3(grid / 2, (mt + 1) / 2), dim3(128), 0, st, a, kb_per_item, grid);
   }
   cudaError_t e = launch_pdl(gemm_weights_m_kernel<false>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
                              kb_per_item);
   if (e != cudaSuccess || !a.tail) return e;
-  return launch_pdl(tail_fixup_kernel<false>, dim3(grid / 2), dim3(128), 0, st, a, kb_per_item, grid);
+  return launch_pdl(tail_fixup_kernel<false>, dim3(grid / 2, mt), dim3(128), 0, st, a, kb_per_item, grid);
 }
 
 cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,

@@ -204,14 +204,21 @@ enumerate_kernel(const float* __restrict__ logits, const bf16* __restrict__ Yall
   }
 }
 
-__global__ void reduce_partials_kernel(const float* __restrict__ partial, int nblk, int nC,
-                                       double* __restrict__ loss_sq, float* __restrict__ losses) {
-  const int s = blockIdx.x * blockDim.x + threadIdx.x;
-  if (s >= nC) return;
+// One warp per subset: lane i adds blocks i, i+32, ... in order, then a fixed shuffle tree;
+// the order depends only on the number of blocks, so the result is reproducible.
+__global__ void __launch_bounds__(32)
+reduce_partials_kernel(const float* __restrict__ partial, int nblk, int nC,
+                       double* __restrict__ loss_sq, float* __restrict__ losses) {
+  const int s = blockIdx.x;
+  const int lane = threadIdx.x;
   double v = 0.0;
-  for (int b = 0; b < nblk; ++b) v += (double)partial[(size_t)b * nC + s];
-  loss_sq[s] = v;
-  losses[s] = (float)sqrt(v);
+  for (int b = lane; b < nblk; b += 32) v += (double)partial[(size_t)b * nC + s];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if (lane == 0) {
+    loss_sq[s] = v;
+    losses[s] = (float)sqrt(v);
+  }
 }
 
 int warps_for(int nC) { return nC <= 2048 ? 4 : 1; }
@@ -244,7 +251,7 @@ cudaError_t launch_enumerate(const float* logits, const bf16* Yall, int T, int E
   enumerate_kernel<<<nblk, nw * 32, smem, st>>>(logits, Yall, T, E, r, h, subsets, nC, partial, Fref, src);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  reduce_partials_kernel<<<(nC + 127) / 128, 128, 0, st>>>(partial, nblk, nC, loss_sq, losses);
+  reduce_partials_kernel<<<nC, 32, 0, st>>>(partial, nblk, nC, loss_sq, losses);
   return cudaGetLastError();
 }
 
