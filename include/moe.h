@@ -116,6 +116,15 @@ int moe_forward_topk(moe_layer_t* layer, const void* x, int T, int k, float beta
                      int32_t* idx_out, float* wn_out, int32_t* n_active_out);
 
 /*
+ * Distance between a token's two selected expert outputs,
+ *   dist[t] = || E_e0(x_t) - E_e1(x_t) ||_2      (no skipping, kept experts only),
+ * the quantity whose concentration App. A.2 assumes (D ~ const) when it derives
+ * the skipping rule; for k = 2 the error of skipping token t is exactly
+ * w~_e1 * dist[t].  x [T][h] bf16 device, dist [T] fp32 device.  Asynchronous.
+ */
+int moe_top2_distance(moe_layer_t* layer, const void* x, int T, float* dist);
+
+/*
  * moe_forward with HOST buffers: copies x_host to the device, runs the layer,
  * copies y back and waits for it.  x_host/y_host [T][h] bf16; pinned memory
  * makes the copies asynchronous to the host but is not required.

@@ -303,6 +303,40 @@ int oracle_moe_forward(const uint16_t *x, const uint16_t *Wg, const uint16_t *W1
   return 0;
 }
 
+/* D_t = || E_e0(x_t) - E_e1(x_t) ||_2 over the token's two selected (kept) experts, the
+ * quantity App. A.2 observes to be concentrated and replaces by a constant D. */
+int oracle_top2_distance(const uint16_t *x, const uint16_t *Wg, const uint16_t *W1,
+                         const uint16_t *W3, const uint16_t *W2, int T, int h, int f, int E,
+                         uint32_t kept_mask, double *dist) {
+  if (E < 2 || E > ORACLE_MAX_E || popcount32(kept_mask & ((1u << E) - 1u)) < 2) return -1;
+#pragma omp parallel
+  {
+    float *a = (float *)malloc(sizeof(float) * (size_t)f);
+    double *o0 = (double *)malloc(sizeof(double) * (size_t)h);
+    double *o1 = (double *)malloc(sizeof(double) * (size_t)h);
+#pragma omp for schedule(dynamic, 1)
+    for (int t = 0; t < T; ++t) {
+      const uint16_t *xt = x + (size_t)t * h;
+      float l[ORACLE_MAX_E], wr[2], wnn[2], rt;
+      int32_t id[2];
+      uint8_t sk;
+      router_logits(xt, Wg, h, E, l);
+      route_token(l, E, kept_mask, 0.0f, id, wr, wnn, &rt, &sk);
+      expert_ffn(xt, W1 + (size_t)id[0] * f * h, W3 + (size_t)id[0] * f * h, W2 + (size_t)id[0] * h * f,
+                 h, f, o0, a);
+      expert_ffn(xt, W1 + (size_t)id[1] * f * h, W3 + (size_t)id[1] * f * h, W2 + (size_t)id[1] * h * f,
+                 h, f, o1, a);
+      double s2 = 0.0;
+      for (int i = 0; i < h; ++i) s2 += (o0[i] - o1[i]) * (o0[i] - o1[i]);
+      dist[t] = sqrt(s2);
+    }
+    free(a);
+    free(o0);
+    free(o1);
+  }
+  return 0;
+}
+
 /* ------------------------------------------------------- top-k generalisation */
 
 /* Routing of one token in the general top-k setting (App. A.2).  e_0..e_{k-1} are the kept

@@ -175,6 +175,24 @@ def frequency_subset(counts, r: int) -> int:
     return int(fn(_p(counts, _i64p), E, r))
 
 
+def top2_distance(x, Wg, W1, W3, W2, kept_mask: int) -> np.ndarray:
+    """dist[T] float64: ||E_e0(x) - E_e1(x)||_2 over each token's two selected experts."""
+    x = _u16(x)
+    T, h = x.shape
+    Wg = _u16(Wg)
+    E = Wg.shape[0]
+    W1 = _u16(W1)
+    f = W1.shape[1]
+    W3 = _u16(W3, (E, f, h))
+    W2 = _u16(W2, (E, h, f))
+    dist = np.zeros(T, np.float64)
+    rc = lib().oracle_top2_distance(_p(x, _u16p), _p(Wg, _u16p), _p(W1, _u16p), _p(W3, _u16p),
+                                    _p(W2, _u16p), T, h, f, E, ctypes.c_uint32(kept_mask), _p(dist, _f64p))
+    if rc:
+        raise ValueError("oracle_top2_distance: invalid arguments")
+    return dist
+
+
 def moe_forward_topk(x, Wg, W1, W3, W2, kept_mask: int, k: int, beta: float):
     """Top-k layer forward with the generalised skipping rule.  Returns dict(y, z, idx[T,k],
     wn[T,k], n_active[T], tail_frac[T], logits[T,E])."""

@@ -54,6 +54,7 @@ def load_library(path: str | None = None):
     lib.moe_forward.argtypes = [vp, vp, ci, cf, vp, vp]
     lib.moe_forward_residual.argtypes = [vp, vp, ci, cf, vp, vp, vp]
     lib.moe_forward_host.argtypes = [vp, vp, ci, cf, vp]
+    lib.moe_top2_distance.argtypes = [vp, vp, ci, vp]
     lib.moe_forward_topk.argtypes = [vp, vp, ci, ci, cf, vp, vp, vp, vp]
     lib.moe_routing_stats_layout.restype = ctypes.c_size_t
     lib.moe_routing_stats_layout.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_size_t)]
@@ -201,6 +202,14 @@ class MoeLayer:
             idx.data_ptr() if record else None, wn.data_ptr() if record else None,
             na.data_ptr() if record else None))
         return (y, idx, wn, na) if record else y
+
+    def top2_distance(self, x):
+        """``moe_top2_distance``: fp32 CUDA tensor [T] of ||E_e0(x) - E_e1(x)||_2."""
+        T = x.shape[0]
+        _dev_bf16(x, (T, self.h))
+        out = torch.empty((T,), dtype=torch.float32, device=x.device)
+        _check(load_library().moe_top2_distance(self._h, x.data_ptr(), T, out.data_ptr()))
+        return out
 
     def forward_host(self, x_host: torch.Tensor, beta: float, y_host: torch.Tensor):
         """``moe_forward_host``: x_host, y_host are host bf16 tensors (pinned or not)."""

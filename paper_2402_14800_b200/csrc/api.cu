@@ -242,12 +242,13 @@ int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmM
   return MOE_OK;
 }
 
+// dist != nullptr: instead of combining, write || E_e0(x) - E_e1(x) ||_2 per token (y unused)
 int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* residual, void* y,
-                 void* stats) {
+                 void* stats, float* dist = nullptr) {
   if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
   if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
   if (T == 0) return MOE_OK;
-  if (!x || !y) return fail(MOE_ERR_INVALID_ARG, "x or y is NULL");
+  if (!x || (!y && !dist)) return fail(MOE_ERR_INVALID_ARG, "x or the output is NULL");
   if (!aligned16(x) || !aligned16(y) || !aligned16(residual) || !aligned16(stats))
     return fail(MOE_ERR_INVALID_ARG, "x, y, residual and routing_stats must be 16-byte aligned");
   if (!(beta >= 0.f)) return fail(MOE_ERR_INVALID_ARG, "beta must be >= 0");
@@ -311,8 +312,12 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
                         (const bf16*)L->ws->act.p, rows_cap, T);
   if (rc) return rc;
   mark(L);
-  CUDA_TRY(launch_combine((const float*)L->ws->O.p, ksplit, split_stride, (int32_t*)L->ws->pair_pos.p,
-                          (float*)L->ws->wn.p, (const bf16*)residual, T, L->h, (bf16*)y, st));
+  if (dist)
+    CUDA_TRY(launch_top2_distance((const float*)L->ws->O.p, ksplit, split_stride,
+                                  (int32_t*)L->ws->pair_pos.p, T, L->h, dist, st));
+  else
+    CUDA_TRY(launch_combine((const float*)L->ws->O.p, ksplit, split_stride, (int32_t*)L->ws->pair_pos.p,
+                            (float*)L->ws->wn.p, (const bf16*)residual, T, L->h, (bf16*)y, st));
   mark(L);
   return MOE_OK;
 }
@@ -458,6 +463,11 @@ int moe_forward(moe_layer_t* L, const void* x, int T, float beta, void* y, void*
 int moe_forward_residual(moe_layer_t* L, const void* x, int T, float beta, const void* residual,
                          void* y, void* routing_stats) {
   return forward_impl(L, x, T, beta, residual, y, routing_stats);
+}
+
+int moe_top2_distance(moe_layer_t* L, const void* x, int T, float* dist) {
+  if (!dist) return fail(MOE_ERR_INVALID_ARG, "dist is NULL");
+  return forward_impl(L, x, T, 0.f, nullptr, nullptr, nullptr, dist);
 }
 
 int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, void* y,

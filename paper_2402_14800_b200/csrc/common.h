@@ -118,6 +118,8 @@ cudaError_t launch_combine_topk(const float* O, int ksplit, size_t split_stride,
                                 bf16* y, cudaStream_t st);
 cudaError_t launch_coselection(const int32_t* idx, int T, int E, const KeptIds& kept, int32_t* counts,
                                cudaStream_t st);
+cudaError_t launch_top2_distance(const float* O, int ksplit, size_t split_stride,
+                                 const int32_t* pair_pos, int T, int h, float* dist, cudaStream_t st);
 cudaError_t launch_rmsnorm(const bf16* x, int T, int h, float eps, bf16* out, cudaStream_t st);
 cudaError_t launch_set_dense_meta(Meta* meta, int E, int rows_per_expert, int off_stride,
                                   cudaStream_t st);

@@ -625,6 +625,40 @@ coselection_kernel(const int32_t* __restrict__ idx, int T, int E, KeptIds kept,
   }
 }
 
+// ------------------------------------------------------------------------- top-2 distance
+
+// D_t = || E_e0(x_t) - E_e1(x_t) ||_2, the quantity App. A.2 observes to be concentrated.
+__global__ void __launch_bounds__(256)
+top2_distance_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
+                     const int32_t* __restrict__ pair_pos, int T, int h, float* __restrict__ dist) {
+  __shared__ float s_part[8];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int t = blockIdx.x;
+  const int p0 = pair_pos[2 * t], p1 = pair_pos[2 * t + 1];
+  float acc = 0.f;
+  if (p1 >= 0) {
+    for (int i = threadIdx.x; i < h; i += blockDim.x) {
+      float a = 0.f, b = 0.f;
+      for (int s = 0; s < ksplit; ++s) {
+        a += O[s * split_stride + (size_t)p0 * h + i];
+        b += O[s * split_stride + (size_t)p1 * h + i];
+      }
+      const float d = a - b;
+      acc = fmaf(d, d, acc);
+    }
+  }
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+    for (int w = 0; w < 8; ++w) tot += s_part[w];
+    dist[t] = sqrtf(tot);
+  }
+}
+
 // ------------------------------------------------------------------------------- rmsnorm
 
 __global__ void __launch_bounds__(256)
@@ -859,6 +893,12 @@ cudaError_t launch_coselection(const int32_t* idx, int T, int E, const KeptIds& 
   if (blocks > 148 * 4) blocks = 148 * 4;
   coselection_kernel<<<blocks, 256, 0, st>>>(idx, T, E, kept, counts);
   return cudaGetLastError();
+}
+
+cudaError_t launch_top2_distance(const float* O, int ksplit, size_t split_stride,
+                                 const int32_t* pair_pos, int T, int h, float* dist, cudaStream_t st) {
+  return launch_pdl(top2_distance_kernel, dim3(T), dim3(256), 0, st, O, ksplit, split_stride, pair_pos,
+                    T, h, dist);
 }
 
 cudaError_t launch_rmsnorm(const bf16* x, int T, int h, float eps, bf16* out, cudaStream_t st) {

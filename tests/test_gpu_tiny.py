@@ -339,3 +339,16 @@ def test_forward_topk_generalised_skipping(E_, kept, k, T, beta):
     np.testing.assert_allclose(wn[both], ora["wn"][both], rtol=2e-5, atol=1e-7)
     P.check_outputs(b(y), ora["y"], both)
     layer.close()
+
+
+@pytest.mark.parametrize("T,kept", [(256, FULL), (1000, 0b11011101), (5, FULL)])
+def test_top2_distance(setup, T, kept):
+    host, dev = setup
+    x = synth.make_tokens(T, H, seed=13)
+    want = O.top2_distance(synth.bf16_bits(x), host["Wg"], host["W1"], host["W3"], host["W2"], kept)
+    tie = P.near_tie_tokens(O.route(synth.bf16_bits(x), host["Wg"], kept, 0.0)["logits"], kept)
+    layer = make_layer(dev, kept)
+    got = layer.top2_distance(x.to(DEV)).cpu().numpy().astype(np.float64)
+    layer.close()
+    ok = ~tie
+    np.testing.assert_allclose(got[ok], want[ok], rtol=5e-3)

@@ -486,3 +486,21 @@ def test_topk_pruned_experts_are_never_selected(cfg16):
     assert all((kept >> int(e)) & 1 for e in out["idx"].ravel())
     with pytest.raises(ValueError):
         fwdk(c, 0b111, 4, 0.0)
+
+
+# ----------------------------------------------------- expert-output distance (App. A.2)
+
+@pytest.mark.parametrize("kept", [FULL, 0b10110110])
+def test_top2_distance_and_exact_skip_error(cfg0, dense, kept):
+    """D_t = ||f_e0 - f_e1|| against the dense numpy outputs; for k = 2 the appendix' bound is an
+    equality: ||z^ - z|| = w~_e1 D_t."""
+    d = O.top2_distance(cfg0["x"], cfg0["Wg"], cfg0["W1"], cfg0["W3"], cfg0["W2"], kept)
+    a = fwd(cfg0, kept=kept, beta=0.0)
+    t = np.arange(T)
+    want = np.linalg.norm(dense["Y"][t, a["idx"][:, 0]] - dense["Y"][t, a["idx"][:, 1]], axis=1)
+    np.testing.assert_allclose(d, want, rtol=1e-9)
+    b = fwd(cfg0, kept=kept, beta=2.0)
+    err = np.linalg.norm(b["z"] - a["z"], axis=1)
+    # the two fp32 weights sum to 1 only up to one rounding, hence the absolute term
+    np.testing.assert_allclose(err, a["wn"][:, 1] * d, rtol=2e-6,
+                               atol=3e-7 * np.linalg.norm(dense["Y"], axis=2).max())
