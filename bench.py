@@ -429,6 +429,11 @@ def run_ours(a):
                                      "random_mean_loss": float(np.mean(losses)),
                                      "worst_loss": max(losses)}
 
+        # concentration of ||f_e0 - f_e1|| that the appendix' derivation of the skipping rule assumes
+        d = layer.top2_distance(x[:min(T, 8192)].contiguous()).double()
+        baselines["top2_distance"] = {"tokens": int(d.numel()), "mean": float(d.mean()),
+                                      "std_over_mean": float(d.std() / d.mean())}
+
     if rank == 0:
         metric, unit = metric_unit(a)
         gpu_launches = launches_per_step * a.steps if launches_per_step else None
