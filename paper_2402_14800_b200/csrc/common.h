@@ -174,6 +174,8 @@ cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& 
 cudaError_t launch_simt_down(const bf16* A, const bf16* W2, const GemmArgs& a, int cap_rows,
                              GemmOut out_kind, cudaStream_t st);
 cudaError_t gemm_set_attributes();
+// token-major GEMMs on CTA pairs (cta_group::2) instead of single CTAs
+void gemm_set_pair_mode(bool on);
 
 // ---- search (search.cu) ---------------------------------------------------------------
 // Where the enumeration finds the expert outputs.  Dense (topk_idx == null): Yall[T][E][h].
