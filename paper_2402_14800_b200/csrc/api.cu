@@ -304,8 +304,8 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;
   GemmMaps m_gu, m_dn;
-  m_gu.w = wm ? L->w13_128 : L->w13_256;
-  m_dn.w = wm ? L->w2_128 : L->w2_256;
+  m_gu.w = (wm || gemm_pair_mode()) ? L->w13_128 : L->w13_256;
+  m_dn.w = (wm || gemm_pair_mode()) ? L->w2_128 : L->w2_256;
   memcpy(m_gu.t, L->ws->tok_x, sizeof(m_gu.t));
   memcpy(m_dn.t, L->ws->tok_act, sizeof(m_dn.t));
   rc = run_expert_gemms(L, meta, wm, m_gu, m_dn, gu, dn, kOutF32, (const bf16*)L->ws->xperm.p,
@@ -517,8 +517,8 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;
   GemmMaps m_gu, m_dn;
-  m_gu.w = wm ? L->w13_128 : L->w13_256;
-  m_dn.w = wm ? L->w2_128 : L->w2_256;
+  m_gu.w = (wm || gemm_pair_mode()) ? L->w13_128 : L->w13_256;
+  m_dn.w = (wm || gemm_pair_mode()) ? L->w2_128 : L->w2_256;
   memcpy(m_gu.t, W.tok_x, sizeof(m_gu.t));
   memcpy(m_dn.t, W.tok_act, sizeof(m_dn.t));
   const bool prof_saved = L->prof;
@@ -662,8 +662,8 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
   L->prof = false;  // stage marks describe moe_forward only
   EnumSource src = {nullptr, nullptr, 0, 0};
   GemmMaps m_gu, m_dn;
-  m_gu.w = L->w13_256;
-  m_dn.w = L->w2_256;
+  m_gu.w = gemm_pair_mode() ? L->w13_128 : L->w13_256;
+  m_dn.w = gemm_pair_mode() ? L->w2_128 : L->w2_256;
 
   if (pruned_work) {
     const int rows_chunk = (int)align_up((size_t)K * Tc + (size_t)E * kTileRows, kTileRows);

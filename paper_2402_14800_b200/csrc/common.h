@@ -176,6 +176,7 @@ cudaError_t launch_simt_down(const bf16* A, const bf16* W2, const GemmArgs& a, i
 cudaError_t gemm_set_attributes();
 // token-major GEMMs on CTA pairs (cta_group::2) instead of single CTAs
 void gemm_set_pair_mode(bool on);
+bool gemm_pair_mode();  // pair mode takes the weight maps with 128-row boxes (each CTA loads half a tile)
 
 // ---- search (search.cu) ---------------------------------------------------------------
 // Where the enumeration finds the expert outputs.  Dense (topk_idx == null): Yall[T][E][h].

@@ -1160,6 +1160,7 @@ static cudaError_t launch_pair(void (*kernel)(KArgs...), int grid, size_t smem, 
 
 static bool g_pair_mode = false;
 void gemm_set_pair_mode(bool on) { g_pair_mode = on; }
+bool gemm_pair_mode() { return g_pair_mode; }
 
 cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps& maps,
                                  const GemmArgs& a, cudaStream_t st) {

@@ -1,0 +1,115 @@
+"""Alternative code paths behind switches, checked against the default path on the GPU:
+the CUDA-core debug kernels, the dense (all experts) search, the CTA-pair token-major GEMM,
+and replay of a captured CUDA graph of moe_forward."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2402_14800_b200 import binding, build, synth
+
+pytestmark = pytest.mark.gpu
+
+H, F, E = 128, 448, 8
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def weights():
+    build.build()
+    W = synth.make_layer_weights(H, F, E, seed=0)
+    return [t.to(DEV) for t in (W.W_gate, W.W1, W.W3, W.W2)]
+
+
+def layer_with_env(weights, kept=0xFF, **env):
+    """The switches are read when a handle is created."""
+    old = {k: os.environ.get(k) for k in env}
+    os.environ.update({k: str(v) for k, v in env.items()})
+    try:
+        return binding.MoeLayer(*weights, kept)
+    finally:
+        for k, v in old.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+
+
+def rel_l2(a, b):
+    """Worst per-token relative L2 distance between two bf16 outputs."""
+    a, b = a.double().cpu().numpy(), b.double().cpu().numpy()
+    return float((np.linalg.norm(a - b, axis=1) / np.linalg.norm(b, axis=1)).max())
+
+
+@pytest.mark.parametrize("T", [40, 700])
+def test_debug_cuda_core_kernels_agree_with_tensor_core_path(weights, T):
+    x = synth.make_tokens(T, H, seed=3).to(DEV)
+    ref = binding.MoeLayer(*weights, 0b11011101)
+    dbg = layer_with_env(weights, 0b11011101, MOE_DEBUG_SIMT=1)
+    y0, y1 = ref.forward(x, 0.4), dbg.forward(x, 0.4)
+    torch.cuda.synchronize()
+    assert rel_l2(y1, y0) < 5e-3  # different summation orders, same rounding points
+    ref.close()
+    dbg.close()
+
+
+@pytest.mark.parametrize("r", [6, 4, 7])
+def test_dense_search_equals_pruned_work_search(weights, r):
+    x = synth.make_tokens(777, H, seed=4).to(DEV)
+    fast = binding.MoeLayer(*weights)
+    dense = layer_with_env(weights, MOE_SEARCH_DENSE=1)
+    l0, b0 = fast.prune_search(x, r)
+    l1, b1 = dense.prune_search(x, r)
+    fast.close()
+    dense.close()
+    np.testing.assert_allclose(l0, l1, rtol=1e-6)
+    assert b0 == b1
+
+
+def test_cta_pair_gemm_agrees_with_single_cta_gemm(weights):
+    x = synth.make_tokens(1500, H, seed=5).to(DEV)
+    one = binding.MoeLayer(*weights)
+    y0 = one.forward(x, 0.3).clone()
+    l0, b0 = one.prune_search(x, 6)
+    one.close()
+    pair = layer_with_env(weights, MOE_GEMM_PAIR=1)
+    try:
+        y1 = pair.forward(x, 0.3)
+        l1, b1 = pair.prune_search(x, 6)
+        torch.cuda.synchronize()
+        assert pair.device_status() == 0
+    finally:
+        pair.close()
+        layer_with_env(weights, MOE_GEMM_PAIR=0).close()  # back to single CTAs for later tests
+    assert rel_l2(y1, y0) < 5e-3
+    np.testing.assert_allclose(l0, l1, rtol=1e-5)
+    assert b0 == b1
+
+
+@pytest.mark.parametrize("T", [16, 600])
+def test_forward_replays_from_a_cuda_graph(weights, T):
+    layer = binding.MoeLayer(*weights)
+    x = synth.make_tokens(T, H, seed=6).to(DEV)
+    y = torch.empty_like(x)
+    s = torch.cuda.Stream(DEV)
+    layer.set_stream(s)
+    with torch.cuda.stream(s):
+        layer.forward(x, 0.4, y=y)          # first call grows the scratch, outside the capture
+        s.synchronize()
+        want = y.clone()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            layer.forward(x, 0.4, y=y)
+        x2 = synth.make_tokens(T, H, seed=7).to(DEV)
+        y.zero_()
+        g.replay()
+        s.synchronize()
+        assert torch.equal(y, want)
+        x.copy_(x2)                          # same buffers, new contents
+        g.replay()
+        s.synchronize()
+        fresh = layer.forward(x2, 0.4)
+        s.synchronize()
+        assert torch.equal(y, fresh)
+    layer.close()
