@@ -1,0 +1,73 @@
+"""Randomised properties of the oracle (hypothesis): invariants that must hold for any shape,
+kept set and beta, checked on small random layers."""
+import numpy as np
+from hypothesis import given, settings, strategies as st
+
+from oracle import moe_oracle as O
+from paper_2402_14800_b200 import synth
+
+
+def layer(h, f, E, T, seed):
+    W = synth.make_layer_weights(h, f, E, seed=seed)
+    x = synth.make_tokens(T, h, seed=seed + 1)
+    b = synth.bf16_bits
+    return dict(x=b(x), Wg=b(W.W_gate), W1=b(W.W1), W3=b(W.W3), W2=b(W.W2))
+
+
+masks = st.integers(min_value=0, max_value=255).filter(lambda m: bin(m).count("1") >= 2)
+
+
+@settings(max_examples=25, deadline=None)
+@given(seed=st.integers(0, 10_000), kept=masks, beta=st.floats(0.0, 1.5))
+def test_forward_invariants(seed, kept, beta):
+    c = layer(64, 64, 8, 24, seed)
+    o = O.moe_forward(c["x"], c["Wg"], c["W1"], c["W3"], c["W2"], kept, beta)
+    # experts come from the kept set, are distinct, and the weights are a convex combination
+    assert all((kept >> int(e)) & 1 for e in o["idx"].ravel())
+    assert (o["idx"][:, 0] != o["idx"][:, 1]).all()
+    np.testing.assert_allclose(o["wn"].sum(1), 1.0, rtol=1e-6)
+    assert (o["wn"][:, 0] >= o["wn"][:, 1]).all() and (o["wn"] >= 0).all()
+    # the skip decision is the strict comparison of the reported ratio with beta
+    assert np.array_equal(o["skipped"].astype(bool), o["ratio"] < np.float32(beta))
+    assert ((o["wn"][:, 1] == 0) == o["skipped"].astype(bool)).all()
+    assert (o["ratio"] <= 1.0).all() and (o["ratio"] > 0).all()
+    # raising beta can only skip more tokens; the kept routing is untouched by beta
+    o2 = O.moe_forward(c["x"], c["Wg"], c["W1"], c["W3"], c["W2"], kept, beta + 0.25)
+    assert (o2["skipped"] >= o["skipped"]).all() and np.array_equal(o2["idx"], o["idx"])
+
+
+@settings(max_examples=10, deadline=None)
+@given(seed=st.integers(0, 10_000), r=st.integers(2, 8))
+def test_search_invariants(seed, r):
+    c = layer(64, 64, 8, 20, seed)
+    s = O.prune_search_allexperts(c["x"], c["Wg"], c["W1"], c["W3"], c["W2"], r)
+    idx = O.route(c["x"], c["Wg"], 0xFF, 0.0)["idx"]
+    pair = (1 << idx[:, 0]) | (1 << idx[:, 1])
+    for C, n, loss in zip(s["subsets"], s["n_changed"], s["losses"]):
+        assert bin(int(C)).count("1") == r
+        assert n == int(((pair & ~int(C)) != 0).sum())
+        assert (loss == 0.0) == (n == 0)
+    assert s["best_subset"] == int(s["subsets"][int(np.argmin(s["losses"]))])
+    # a superset of experts never disturbs more tokens than its subset
+    if r < 8:
+        big = O.prune_search_allexperts(c["x"], c["Wg"], c["W1"], c["W3"], c["W2"], r + 1)
+        lookup = {int(C): n for C, n in zip(big["subsets"], big["n_changed"])}
+        for C, n in zip(s["subsets"], s["n_changed"]):
+            for e in range(8):
+                if not (int(C) >> e) & 1:
+                    assert lookup[int(C) | (1 << e)] <= n
+
+
+@settings(max_examples=15, deadline=None)
+@given(seed=st.integers(0, 10_000), k=st.integers(1, 6), beta=st.floats(0.0, 1.0))
+def test_topk_invariants(seed, k, beta):
+    c = layer(64, 64, 8, 16, seed)
+    o = O.moe_forward_topk(c["x"], c["Wg"], c["W1"], c["W3"], c["W2"], 0xFF, k, beta)
+    assert ((o["n_active"] >= 1) & (o["n_active"] <= k)).all()
+    for t in range(16):
+        assert len(set(o["idx"][t].tolist())) == k
+        l = o["logits"][t][o["idx"][t]]
+        assert (np.diff(l) <= 0).all()                      # decreasing routing weight
+        assert (o["wn"][t, o["n_active"][t]:] == 0).all() and (o["wn"][t, :o["n_active"][t]] > 0).all()
+    np.testing.assert_allclose(o["wn"].sum(1), 1.0, rtol=1e-6)
+    assert (o["tail_frac"] <= beta + 1e-6).all()
