@@ -42,14 +42,22 @@ def measured_peaks():
     return dict(hbm=6650.0, tf_burst=1590.0, tf_sust=1400.0, source="fallback")
 
 
+def kernel_source_sha256(kernel: str):
+    """Hash of the source text of one __global__ kernel in csrc/gemm_sm100.cu (from its name to
+    the closing brace in column 0)."""
+    import hashlib
+    src = open(os.path.join(ROOT, "paper_2402_14800_b200", "csrc", "gemm_sm100.cu")).read()
+    i = src.index("\n" + kernel + "(")
+    j = src.index("\n}\n", i)
+    return hashlib.sha256(src[i:j].encode()).hexdigest()
+
+
 def recorded_traffic(workload: str):
     """DRAM bytes per launch of the dominant kernel from the committed ncu capture of this
-    workload, or None when there is none or the kernel source changed since."""
-    import hashlib
+    workload, or None when there is none or that kernel's source changed since."""
     try:
         rec = json.load(open(os.path.join(ROOT, "profiles", "traffic.json"))).get(workload)
-        src = os.path.join(ROOT, "paper_2402_14800_b200", "csrc", "gemm_sm100.cu")
-        if rec and hashlib.sha256(open(src, "rb").read()).hexdigest() == rec["kernel_source_sha256"]:
+        if rec and kernel_source_sha256(rec["kernel_function"]) == rec["kernel_source_sha256"]:
             return rec["dram_bytes"]
     except Exception:
         pass
