@@ -279,8 +279,9 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   mark(L);
   if (dec) {
     CUDA_TRY(launch_router_small((const bf16*)x, L->Wg, T, L->h, L->r, beta, L->kept, ro, st));
-    CUDA_TRY(launch_permute_small(ro.idx, ro.skipped, T, L->r, 16, meta, (int32_t*)L->ws->pair_pos.p,
-                                  (int32_t*)L->ws->row_token.p, s_count, s_nsk, s_nt, L->kept, L->E, st));
+    CUDA_TRY(launch_permute_gather_small((const bf16*)x, ro.idx, ro.skipped, T, L->h, L->r, 16, meta,
+                                         (int32_t*)L->ws->pair_pos.p, (int32_t*)L->ws->row_token.p,
+                                         (bf16*)L->ws->xperm.p, s_count, s_nsk, s_nt, L->kept, L->E, st));
   } else {
     CUDA_TRY(launch_router((const bf16*)x, L->Wg, T, L->h, L->r, beta, L->kept, ro, st));
     CUDA_TRY(launch_scan(ro.blk_hist, nblk, L->r, kTileRows, (int32_t*)L->ws->blk_base.p, meta,
@@ -289,8 +290,9 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
     CUDA_TRY(launch_scatter(ro.idx, ro.skipped, (int32_t*)L->ws->blk_base.p, meta, T,
                             (int32_t*)L->ws->pair_pos.p, (int32_t*)L->ws->row_token.p, st));
   }
-  CUDA_TRY(launch_gather((const bf16*)x, (int32_t*)L->ws->row_token.p, meta, L->h, rows_cap,
-                         (bf16*)L->ws->xperm.p, st));
+  if (!dec)
+    CUDA_TRY(launch_gather((const bf16*)x, (int32_t*)L->ws->row_token.p, meta, L->h, rows_cap,
+                           (bf16*)L->ws->xperm.p, st));
   mark(L);
 
   GemmArgs gu, dn;

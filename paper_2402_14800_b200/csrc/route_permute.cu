@@ -120,90 +120,106 @@ router_small_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
   }
 }
 
-// Small batches: the whole permutation in one block (histogram, offsets, ranks, scatter and
-// the padding rows), T <= blockDim.x.
+// Small batches: permutation and gather in one launch, one block per token.  Every block
+// recomputes the (tiny) histogram and offsets from the routing record, places its own token's
+// pairs and copies the token's row to them; block 0 also publishes the batch description.
+// Padding rows of the groups are left as they are: in the weight-major GEMM a token row only
+// feeds its own accumulator column, and the columns of padding rows are never stored.
 __global__ void __launch_bounds__(kDecodeMaxT)
-permute_small_kernel(const int32_t* __restrict__ idx, const uint8_t* __restrict__ skipped, int T,
-                     int r, int pad, Meta* meta, int32_t* __restrict__ pair_pos,
-                     int32_t* __restrict__ row_token, int32_t* s_count, int32_t* s_nskipped,
-                     int32_t* s_ntouched, KeptIds kept, int E) {
+permute_gather_small_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ idx,
+                            const uint8_t* __restrict__ skipped, int T, int h, int r, int pad,
+                            Meta* meta, int32_t* __restrict__ pair_pos,
+                            int32_t* __restrict__ row_token, bf16* __restrict__ xperm,
+                            int32_t* s_count, int32_t* s_nskipped, int32_t* s_ntouched, KeptIds kept,
+                            int E) {
   pdl_launch_dependents();
   pdl_wait();
   __shared__ int s_e[kDecodeMaxT][2];
   __shared__ int s_cnt[kMaxE][2];
   __shared__ int s_off[kMaxE + 1];
   __shared__ int s_nsk;
-  const int t = threadIdx.x;
-  int e0 = -1, e1 = -1;
-  if (t < T) {
-    e0 = idx[2 * t];
-    e1 = skipped[t] ? -1 : idx[2 * t + 1];
+  __shared__ int s_p[2];
+  const int i = threadIdx.x;
+  const int t = blockIdx.x;
+  {
+    int e0 = -1, e1 = -1;
+    if (i < T) {
+      e0 = idx[2 * i];
+      e1 = skipped[i] ? -1 : idx[2 * i + 1];
+    }
+    s_e[i][0] = e0;
+    s_e[i][1] = e1;
   }
-  s_e[t][0] = e0;
-  s_e[t][1] = e1;
   __syncthreads();
-  if (t < 2 * r) {
-    const int c = t >> 1, slot = t & 1;
+  if (i < 2 * r) {
+    const int c = i >> 1, slot = i & 1;
     int n = 0;
-    for (int i = 0; i < T; ++i) n += (s_e[i][slot] == c);
+    for (int q = 0; q < T; ++q) n += (s_e[q][slot] == c);
     s_cnt[c][slot] = n;
-  } else if (t == 2 * kMaxE) {
+  } else if (i == 2 * kMaxE) {
     int n = 0;
-    for (int i = 0; i < T; ++i) n += (s_e[i][1] < 0);
+    for (int q = 0; q < T; ++q) n += (s_e[q][1] < 0);
     s_nsk = n;
   }
   __syncthreads();
-  if (t == 0) {
+  if (i == 0) {
     int off = 0, tiles = 0, touched = 0;
-    meta->off[0] = 0;
-    meta->tile_prefix[0] = 0;
     s_off[0] = 0;
     for (int c = 0; c < kMaxE; ++c) {
-      const int n0 = c < r ? s_cnt[c][0] : 0, n1 = c < r ? s_cnt[c][1] : 0;
-      const int n = n0 + n1;
-      meta->count[c] = n;
-      meta->count_slot[c][0] = n0;
-      meta->count_slot[c][1] = n1;
+      const int n = c < r ? s_cnt[c][0] + s_cnt[c][1] : 0;
       off += (n + pad - 1) / pad * pad;
       tiles += (n + kTileRows - 1) / kTileRows;
       touched += (n > 0);
-      meta->off[c + 1] = off;
-      meta->tile_prefix[c + 1] = tiles;
       s_off[c + 1] = off;
-    }
-    meta->rows_total = off;
-    meta->n_skipped = s_nsk;
-    meta->n_touched = touched;
-    meta->reserved = 0;
-    if (s_count) {
-      for (int e = 0; e < E; ++e) { s_count[2 * e] = 0; s_count[2 * e + 1] = 0; }
-      for (int c = 0; c < r; ++c) {
-        s_count[2 * kept.id[c]] = s_cnt[c][0];
-        s_count[2 * kept.id[c] + 1] = s_cnt[c][1];
+      if (t == 0) {
+        meta->count[c] = n;
+        meta->count_slot[c][0] = c < r ? s_cnt[c][0] : 0;
+        meta->count_slot[c][1] = c < r ? s_cnt[c][1] : 0;
+        meta->off[c + 1] = off;
+        meta->tile_prefix[c + 1] = tiles;
       }
-      *s_nskipped = s_nsk;
-      *s_ntouched = touched;
+    }
+    if (t == 0) {
+      meta->off[0] = 0;
+      meta->tile_prefix[0] = 0;
+      meta->rows_total = off;
+      meta->n_skipped = s_nsk;
+      meta->n_touched = touched;
+      meta->reserved = 0;
+      if (s_count) {
+        for (int e = 0; e < E; ++e) { s_count[2 * e] = 0; s_count[2 * e + 1] = 0; }
+        for (int c = 0; c < r; ++c) {
+          s_count[2 * kept.id[c]] = s_cnt[c][0];
+          s_count[2 * kept.id[c] + 1] = s_cnt[c][1];
+        }
+        *s_nskipped = s_nsk;
+        *s_ntouched = touched;
+      }
     }
   }
   __syncthreads();
-  if (t < T) {
-    int r0 = 0, r1 = 0;
-    for (int i = 0; i < t; ++i) {
-      r0 += (s_e[i][0] == e0) + (s_e[i][1] == e0);
-      r1 += (s_e[i][0] == e1) + (s_e[i][1] == e1);
+  if (i < 2) {
+    const int c = s_e[t][i];
+    int pos = -1;
+    if (c >= 0) {
+      int rank = 0;
+      for (int q = 0; q < t; ++q) rank += (s_e[q][0] == c) + (s_e[q][1] == c);
+      pos = s_off[c] + rank;
+      row_token[pos] = t;
     }
-    const int p0 = s_off[e0] + r0;
-    row_token[p0] = t;
-    pair_pos[2 * t] = p0;
-    int p1 = -1;
-    if (e1 >= 0) {
-      p1 = s_off[e1] + r1;
-      row_token[p1] = t;
-    }
-    pair_pos[2 * t + 1] = p1;
+    pair_pos[2 * t + i] = pos;
+    s_p[i] = pos;
   }
-  if (t < r) {  // padding rows of this expert's group gather zeros
-    for (int row = s_off[t] + s_cnt[t][0] + s_cnt[t][1]; row < s_off[t + 1]; ++row) row_token[row] = -1;
+  __syncthreads();
+  const int nvec = h >> 3;
+  const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * h);
+  const int p0 = s_p[0], p1 = s_p[1];
+  uint4* d0 = reinterpret_cast<uint4*>(xperm + (size_t)p0 * h);
+  uint4* d1 = reinterpret_cast<uint4*>(xperm + (size_t)(p1 < 0 ? p0 : p1) * h);
+  for (int v = i; v < nvec; v += blockDim.x) {
+    const uint4 val = __ldg(src + v);
+    d0[v] = val;
+    if (p1 >= 0) d1[v] = val;
   }
 }
 
@@ -813,12 +829,13 @@ cudaError_t launch_router_small(const bf16* x, const bf16* Wg, int T, int h, int
   return cudaGetLastError();
 }
 
-cudaError_t launch_permute_small(const int32_t* idx, const uint8_t* skipped, int T, int r, int pad,
-                                 Meta* meta, int32_t* pair_pos, int32_t* row_token,
-                                 int32_t* s_count, int32_t* s_nskipped, int32_t* s_ntouched,
-                                 const KeptIds& kept, int E, cudaStream_t st) {
-  return launch_pdl(permute_small_kernel, dim3(1), dim3(kDecodeMaxT), 0, st, idx, skipped, T, r, pad,
-                    meta, pair_pos, row_token, s_count, s_nskipped, s_ntouched, kept, E);
+cudaError_t launch_permute_gather_small(const bf16* x, const int32_t* idx, const uint8_t* skipped, int T,
+                                        int h, int r, int pad, Meta* meta, int32_t* pair_pos,
+                                        int32_t* row_token, bf16* xperm, int32_t* s_count,
+                                        int32_t* s_nskipped, int32_t* s_ntouched, const KeptIds& kept,
+                                        int E, cudaStream_t st) {
+  return launch_pdl(permute_gather_small_kernel, dim3(T), dim3(kDecodeMaxT), 0, st, x, idx, skipped, T, h,
+                    r, pad, meta, pair_pos, row_token, xperm, s_count, s_nskipped, s_ntouched, kept, E);
 }
 
 cudaError_t launch_scan(const int32_t* blk_hist, int nblk, int r, int pad, int32_t* blk_base,
