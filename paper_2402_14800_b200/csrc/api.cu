@@ -301,7 +301,10 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   gu.a_off_mul = 1; gu.out_off_mul = 1; gu.out_ld = L->f; gu.out = L->ws->act.p;
   dn.a_off_mul = 1; dn.out_off_mul = 1; dn.out_ld = L->h; dn.out = L->ws->O.p;
   const bool wm = dec && !L->debug_simt;
-  if (wm) { gu.tail = (float*)L->ws->tail.p; dn.tail = (float*)L->ws->tail.p; }
+  if (wm) {
+    gu.tail = (float*)L->ws->tail.p; dn.tail = (float*)L->ws->tail.p;
+    gu.tail_info = (int*)L->ws->status.p + 1; dn.tail_info = (int*)L->ws->status.p + 1;
+  }
   const int ksplit = wm ? ksplit_for(L) : 1;
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;
@@ -514,7 +517,10 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
   gu.a_off_mul = 1; gu.out_off_mul = 1; gu.out_ld = L->f; gu.out = W.act.p;
   dn.a_off_mul = 1; dn.out_off_mul = 1; dn.out_ld = L->h; dn.out = W.O.p;
   const bool wm = dec && !L->debug_simt;
-  if (wm) { gu.tail = (float*)W.tail.p; dn.tail = (float*)W.tail.p; }
+  if (wm) {
+    gu.tail = (float*)W.tail.p; dn.tail = (float*)W.tail.p;
+    gu.tail_info = (int*)W.status.p + 1; dn.tail_info = (int*)W.status.p + 1;
+  }
   const int ksplit = wm ? ksplit_for(L) : 1;
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;

@@ -148,6 +148,7 @@ struct GemmArgs {
   long long split_stride;  // elements between split-K partial planes (decode down-proj)
   int* status;             // device error word
   float* tail;             // weight-major kernel: partial tiles of K-sliced tail items, or null
+  int* tail_info;          // [0] = number of K-sliced tail items of the launch before a fix-up
 };
 
 constexpr size_t kTailBufferBytes = (size_t)256 * 128 * 128 * 4;  // one 64 KB slot per CTA

@@ -803,6 +803,7 @@ __device__ __forceinline__ void decode_item_w(const Meta& m, const GemmArgs& a, 
 }
 
 constexpr int kTailSlotFloats = 128 * WM_BN;  // one partial tile: [token][weight row] fp32
+constexpr int kFixupTokens = 2;  // tokens of a tail tile folded by one fix-up block
 
 template <bool GATE_UP>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -832,6 +833,8 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   const SchedW sched = make_sched_w(s_meta, args, kb_per_item, (int)gridDim.x);
   const int n_items = sched.n_total;
   uint32_t issued = 0;
+  // the fix-up launch that follows only needs `rem` blocks: tell it, so the others leave at once
+  if (blockIdx.x == 0 && threadIdx.x == 0 && args.tail_info) args.tail_info[0] = sched.rem;
 
   if (warp == 0) {
     uint32_t it = 0;
@@ -967,48 +970,64 @@ template <bool GATE_UP>
 __global__ void __launch_bounds__(128)
 tail_fixup_kernel(const GemmArgs args, int kb_per_item, int gemm_grid) {
   __shared__ Meta s_meta;
+  __shared__ ItemW s_w;
+  __shared__ int s_nslice, s_kst;
   pdl_launch_dependents();
   pdl_wait();
+  if ((int)blockIdx.x >= args.tail_info[0]) return;  // written by the GEMM this launch follows
   for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
     reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
   __syncthreads();
-  const SchedW sched = make_sched_w(s_meta, args, kb_per_item, gemm_grid);
-  if ((int)blockIdx.x >= sched.rem) return;
-  ItemW w;
-  // slices of this tail item, in slice order; empty slices were never written
-  int nslice = 0;
-  for (int sub = 0; sub < sched.KSt; ++sub) {
-    decode_item_w(s_meta, args, sched, sched.full + (int)blockIdx.x * sched.KSt + sub, w);
-    if (w.kb0 < w.kb1) nslice = sub + 1;
-  }
-  decode_item_w(s_meta, args, sched, sched.full + (int)blockIdx.x * sched.KSt, w);
-  const float* slot0 = args.tail + (size_t)(blockIdx.x * sched.KSt) * kTailSlotFloats;
-  // blockIdx.y walks the tokens of the tile (two per block for gate/up, one for down), so each
-  // thread produces one output from nslice independent loads
-  if (GATE_UP) {
-    // 64 features per tile: rows 32q + s are gate, 32q + 16 + s up
-    const int n = 2 * blockIdx.y + (threadIdx.x >> 6), fj = threadIdx.x & 63;
-    const int q = fj >> 4, sft = fj & 15;
-    if (n >= w.cnt || w.mt * 128 + 32 * q >= args.n_w_rows) return;
-    float g = 0.f, u = 0.f;
-#pragma unroll 4
-    for (int sub = 0; sub < nslice; ++sub) {
-      const float* t = slot0 + (size_t)sub * kTailSlotFloats + n * 128;
-      g += t[32 * q + sft];
-      u += t[32 * q + 16 + sft];
+  if (threadIdx.x == 0) {
+    const SchedW sched = make_sched_w(s_meta, args, kb_per_item, gemm_grid);
+    ItemW w;
+    // slices of this tail item, in slice order; empty slices were never written
+    int nslice = 0;
+    for (int sub = 0; sub < sched.KSt; ++sub) {
+      decode_item_w(s_meta, args, sched, sched.full + (int)blockIdx.x * sched.KSt + sub, w);
+      if (w.kb0 < w.kb1) nslice = sub + 1;
     }
+    decode_item_w(s_meta, args, sched, sched.full + (int)blockIdx.x * sched.KSt, w);
+    s_w = w;
+    s_nslice = nslice;
+    s_kst = sched.KSt;
+  }
+  __syncthreads();
+  const ItemW w = s_w;
+  const int nslice = s_nslice;
+  const float* slot0 = args.tail + (size_t)(blockIdx.x * s_kst) * kTailSlotFloats;
+  // blockIdx.y walks the tokens of the tile in groups of kFixupTokens; every output is the sum
+  // of nslice independent loads
+  const int n_begin = blockIdx.y * kFixupTokens;
+  const int n_end = min(w.cnt, n_begin + kFixupTokens);
+  if (GATE_UP) {
+    // 64 features per tile: rows 32q + s are gate, 32q + 16 + s up; two tokens per pass
+    const int fj = threadIdx.x & 63;
+    const int q = fj >> 4, sft = fj & 15;
+    if (w.mt * 128 + 32 * q >= args.n_w_rows) return;
     const int feat = (w.mt * 4 + q) * kInterleave + sft;
-    reinterpret_cast<bf16*>(args.out)[(long long)(w.out_row + n) * args.out_ld + feat] =
-        __float2bfloat16_rn(silu_mul(g, u));
+    for (int n = n_begin + (threadIdx.x >> 6); n < n_end; n += 2) {
+      float g = 0.f, u = 0.f;
+#pragma unroll 8
+      for (int sub = 0; sub < nslice; ++sub) {
+        const float* t = slot0 + (size_t)sub * kTailSlotFloats + n * 128;
+        g += t[32 * q + sft];
+        u += t[32 * q + 16 + sft];
+      }
+      reinterpret_cast<bf16*>(args.out)[(long long)(w.out_row + n) * args.out_ld + feat] =
+          __float2bfloat16_rn(silu_mul(g, u));
+    }
   } else {
-    const int n = blockIdx.y, col = threadIdx.x;
+    const int col = threadIdx.x;
     const int wrow = w.mt * 128 + col;
-    if (n >= w.cnt || wrow >= args.n_w_rows) return;
-    float v = 0.f;
-#pragma unroll 4
-    for (int sub = 0; sub < nslice; ++sub) v += slot0[(size_t)sub * kTailSlotFloats + n * 128 + col];
-    reinterpret_cast<float*>(args.out)[(long long)w.ks * args.split_stride +
-                                       (long long)(w.out_row + n) * args.out_ld + wrow] = v;
+    if (wrow >= args.n_w_rows) return;
+    for (int n = n_begin; n < n_end; ++n) {
+      float v = 0.f;
+#pragma unroll 8
+      for (int sub = 0; sub < nslice; ++sub) v += slot0[(size_t)sub * kTailSlotFloats + n * 128 + col];
+      reinterpret_cast<float*>(args.out)[(long long)w.ks * args.split_stride +
+                                         (long long)(w.out_row + n) * args.out_ld + wrow] = v;
+    }
   }
 }
 
@@ -1186,12 +1205,12 @@ cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const Gemm
     cudaError_t e = launch_pdl(gemm_weights_m_kernel<true>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
                                kb_per_item);
     if (e != cudaSuccess || !a.tail) return e;
-    return launch_pdl(tail_fixup_kernel<true>, dim3(grid / 2, (mt + 1) / 2), dim3(128), 0, st, a, kb_per_item, grid);
+    return launch_pdl(tail_fixup_kernel<true>, dim3(grid / 2, (mt + kFixupTokens - 1) / kFixupTokens), dim3(128), 0, st, a, kb_per_item, grid);
   }
   cudaError_t e = launch_pdl(gemm_weights_m_kernel<false>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
                              kb_per_item);
   if (e != cudaSuccess || !a.tail) return e;
-  return launch_pdl(tail_fixup_kernel<false>, dim3(grid / 2, mt), dim3(128), 0, st, a, kb_per_item, grid);
+  return launch_pdl(tail_fixup_kernel<false>, dim3(grid / 2, (mt + kFixupTokens - 1) / kFixupTokens), dim3(128), 0, st, a, kb_per_item, grid);
 }
 
 cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,
