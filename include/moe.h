@@ -15,6 +15,7 @@
  *     is asynchronous unless the call returns results to host memory.
  *   - A handle must not be used from two host threads at once: its scratch
  *     buffers are shared by all of its calls.
+ *   - A call takes at most 2^24 tokens.
  */
 #ifndef MOE_H_
 #define MOE_H_

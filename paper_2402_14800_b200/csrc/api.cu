@@ -31,6 +31,7 @@ int fail(int code, const char* fmt, ...) {
                   #expr, cudaGetErrorString(e_));                                        \
   } while (0)
 
+constexpr int kMaxTokens = 1 << 24;  // per call; keeps every row index and byte count in range
 inline int popc(uint32_t v) { return __builtin_popcount(v); }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -246,7 +247,7 @@ int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmM
 int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* residual, void* y,
                  void* stats, float* dist = nullptr) {
   if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
-  if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
+  if (T < 0 || T > kMaxTokens) return fail(MOE_ERR_INVALID_ARG, "T = %d outside 0..%d", T, kMaxTokens);
   if (T == 0) return MOE_OK;
   if (!x || (!y && !dist)) return fail(MOE_ERR_INVALID_ARG, "x or the output is NULL");
   if (!aligned16(x) || !aligned16(y) || !aligned16(residual) || !aligned16(stats))
@@ -480,7 +481,7 @@ int moe_top2_distance(moe_layer_t* L, const void* x, int T, float* dist) {
 int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, void* y,
                      int32_t* idx_out, float* wn_out, int32_t* n_active_out) {
   if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
-  if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
+  if (T < 0 || T > kMaxTokens) return fail(MOE_ERR_INVALID_ARG, "T = %d outside 0..%d", T, kMaxTokens);
   if (k < 1 || k > L->r || k > 8) return fail(MOE_ERR_INVALID_ARG, "k = %d outside 1..min(kept experts, 8)", k);
   if (T == 0) return MOE_OK;
   if (!x || !y || x == y) return fail(MOE_ERR_INVALID_ARG, "x and y must be distinct and non-NULL");
@@ -542,7 +543,7 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
 
 int moe_forward_host(moe_layer_t* L, const void* x_host, int T, float beta, void* y_host) {
   if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
-  if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
+  if (T < 0 || T > kMaxTokens) return fail(MOE_ERR_INVALID_ARG, "T = %d outside 0..%d", T, kMaxTokens);
   if (T == 0) return MOE_OK;
   if (!x_host || !y_host) return fail(MOE_ERR_INVALID_ARG, "x_host or y_host is NULL");
   const size_t bytes = (size_t)T * L->h * 2;
@@ -558,7 +559,8 @@ int moe_forward_host(moe_layer_t* L, const void* x_host, int T, float beta, void
 int moe_calibrate_beta(moe_layer_t* L, const void* x, int T, float* beta_out) {
   if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
   if (!x || !beta_out) return fail(MOE_ERR_INVALID_ARG, "x or beta_out is NULL");
-  if (T < 1) return fail(MOE_ERR_INVALID_ARG, "T = %d: at least one calibration token is needed", T);
+  if (T < 1 || T > kMaxTokens)
+    return fail(MOE_ERR_INVALID_ARG, "T = %d outside 1..%d calibration tokens", T, kMaxTokens);
   if (!aligned16(x)) return fail(MOE_ERR_INVALID_ARG, "x must be 16-byte aligned");
   int rc;
   if ((rc = ensure_route(L, T))) return rc;
@@ -578,7 +580,7 @@ int moe_calibrate_beta(moe_layer_t* L, const void* x, int T, float* beta_out) {
 int moe_coselection(moe_layer_t* L, const void* x, int T, int32_t* counts) {
   if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
   if (!x || !counts) return fail(MOE_ERR_INVALID_ARG, "x or counts is NULL");
-  if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
+  if (T < 0 || T > kMaxTokens) return fail(MOE_ERR_INVALID_ARG, "T = %d outside 0..%d", T, kMaxTokens);
   if (!aligned16(x)) return fail(MOE_ERR_INVALID_ARG, "x must be 16-byte aligned");
   const int E = L->E;
   memset(counts, 0, sizeof(int32_t) * E * E);
@@ -621,7 +623,8 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
   if (!x_calib || !losses || !best_subset)
     return fail(MOE_ERR_INVALID_ARG, "x_calib, losses or best_subset is NULL");
   if (!aligned16(x_calib)) return fail(MOE_ERR_INVALID_ARG, "x_calib must be 16-byte aligned");
-  if (T < 1) return fail(MOE_ERR_INVALID_ARG, "T = %d: at least one calibration token is needed", T);
+  if (T < 1 || T > kMaxTokens)
+    return fail(MOE_ERR_INVALID_ARG, "T = %d outside 1..%d calibration tokens", T, kMaxTokens);
   if (L->r != L->E)
     return fail(MOE_ERR_INVALID_ARG, "the search needs a layer created with all %d experts kept", L->E);
   if (r < 2 || r > L->E) return fail(MOE_ERR_INVALID_ARG, "r = %d outside 2..%d", r, L->E);
@@ -801,7 +804,7 @@ int moe_rmsnorm(const void* x, int T, int h, float eps, void* out, void* cuda_st
 int moe_stack_forward(moe_layer_t* const* layers, int n_layers, const void* x, int T,
                       const float* betas, float eps, void* y) {
   if (!layers || n_layers < 1) return fail(MOE_ERR_INVALID_ARG, "no layers");
-  if (T < 0) return fail(MOE_ERR_INVALID_ARG, "T = %d is negative", T);
+  if (T < 0 || T > kMaxTokens) return fail(MOE_ERR_INVALID_ARG, "T = %d outside 0..%d", T, kMaxTokens);
   if (T == 0) return MOE_OK;
   if (!x || !y || x == y) return fail(MOE_ERR_INVALID_ARG, "x and y must be distinct and non-NULL");
   moe_layer* L0 = layers[0];

@@ -142,6 +142,9 @@ def test_argument_errors(setup):
         layer.forward(x, -1.0)
     with pytest.raises(binding.MoeError):
         layer.forward(x, 0.0, y=x)
+    lib = binding.load_library()
+    assert lib.moe_forward(layer._h, x.data_ptr(), (1 << 24) + 1, 0.0, x.data_ptr(), None) == -1
+    assert lib.moe_forward(layer._h, x.data_ptr(), -3, 0.0, x.data_ptr(), None) == -1
     layer.close()
     full = make_layer(dev)
     for r in (1, 9):
