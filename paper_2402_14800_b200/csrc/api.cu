@@ -390,6 +390,8 @@ moe_layer_t* moe_layer_create(const void* W_gate, const void* W1, const void* W3
   for (int c = L->r; c < kMaxE; ++c) L->kept.id[c] = 0;
   const char* dbg = getenv("MOE_DEBUG_SIMT");
   L->debug_simt = dbg && dbg[0] == '1';
+  const char* nopdl = getenv("MOE_NO_PDL");
+  if (nopdl) g_pdl_enabled = nopdl[0] != '1';
   const char* pair = getenv("MOE_GEMM_PAIR");
   if (pair) gemm_set_pair_mode(pair[0] == '1');
   const char* dense = getenv("MOE_SEARCH_DENSE");
