@@ -37,7 +37,7 @@ def load_library(path: str | None = None):
     global _lib
     if _lib is not None and path is None:
         return _lib
-    p = path or _LIB_PATH
+    p = path or os.environ.get("MOE_LIBRARY") or _LIB_PATH  # MOE_LIBRARY: another build of the library
     if not os.path.exists(p):
         raise MoeError(-3, "%s not found: build it with `python -m paper_2402_14800_b200.build`" % p)
     lib = ctypes.CDLL(p)

@@ -28,7 +28,10 @@ namespace {
 
 constexpr int BK = 64;            // k elements per pipeline stage = one 128-byte swizzle span
 constexpr int UMMA_K = 16;        // k elements per tcgen05.mma (bf16)
-constexpr int kBand = 16;         // row tiles that sweep the weight tiles together (L2 reuse)
+#ifndef MOE_KBAND
+#define MOE_KBAND 16
+#endif
+constexpr int kBand = MOE_KBAND;  // row tiles that sweep the weight tiles together (L2 reuse)
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;
 constexpr unsigned long long kDrainLimitNs = 2000000ull;
 
