@@ -109,6 +109,20 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
       : "memory");
 }
+// the same with an L2 eviction policy (weights that are read exactly once)
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                                 int c2, uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst),
                "r"(ncols)
@@ -725,7 +739,10 @@ gemm_tokens_m2_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
 
 // ----------------------------------------------------------------------- gemm_weights_m
 
-constexpr int WM_NS = 6;
+#ifndef MOE_WM_NS
+#define MOE_WM_NS 6
+#endif
+constexpr int WM_NS = MOE_WM_NS;
 constexpr int WM_A_BYTES = 128 * 128;  // 128 weight rows x 64 bf16
 constexpr int WM_B_BYTES = 128 * 128;  // up to 128 token rows x 64 bf16
 constexpr int WM_STAGE = WM_A_BYTES + WM_B_BYTES;
@@ -843,6 +860,9 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   if (warp == 0) {
     uint32_t it = 0;
     bool ok = true;
+#ifndef MOE_WM_NO_EVICT_FIRST
+    const uint64_t evict_first = l2_policy_evict_first();
+#endif
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
       ItemW w;
       decode_item_w(s_meta, args, sched, item, w);
@@ -856,7 +876,13 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
           const uint32_t full = smem_u32(&bars.full[s]);
           const uint32_t sa = smem_base + s * WM_STAGE;
           mbar_expect_tx(full, bytes);
+#ifndef MOE_WM_NO_EVICT_FIRST
+          // every weight byte is read exactly once: do not let it push the token rows, the
+          // activations and the partial sums out of L2
+          tma_load_3d_hint(sa, &maps.w, kb * BK, w.mt * 128, w.c, full, evict_first);
+#else
           tma_load_3d(sa, &maps.w, kb * BK, w.mt * 128, w.c, full);
+#endif
           tma_load_2d(sa + WM_A_BYTES, &maps.t[w.bucket], kb * BK, w.tok_row, full);
         }
         __syncwarp();
