@@ -377,7 +377,7 @@ def run_ours(a):
                   "combine_ms": stage_ms[3] / ncalls}
         if a.workload == "decode":
             gu_bytes = touched * 2 * F * H * 2 + pairs * H * 2 + pairs * F * 2
-            dn_bytes = touched * H * F * 2 + pairs * F * 2 + 7 * pairs * H * 4
+            dn_bytes = touched * H * F * 2 + pairs * F * 2 + 2 * pairs * H * 4
             ach = gu_bytes / (gu_ms * 1e-3) / 1e9
             roofline = {"bound": "hbm", "kernel": "gemm_weights_m_kernel<gate_up>", "achieved": ach,
                         "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"],

@@ -18,7 +18,10 @@ constexpr int kRouteTokPerBlock = 64;     // tokens routed by one block (8 warps
 constexpr int kHistCols = 2 * kMaxE + 1;  // per (expert, slot) pair counts + skipped count
 constexpr int kInterleave = 16;           // W1/W3 rows are interleaved in groups of 16
 constexpr int kDecodeMaxT = 256;          // up to here the weight-stationary GEMM is used
-constexpr int kDecodeKbPerItem = 32;      // k-blocks (of 64) per split-K item, decode down-proj
+#ifndef MOE_DOWN_KB
+#define MOE_DOWN_KB 112
+#endif
+constexpr int kDecodeKbPerItem = MOE_DOWN_KB;  // k-blocks (of 64) per split-K item, decode down-proj
 
 // Device-resident description of one permuted batch, written by the scan kernel
 // (or by set_dense_meta for the search) and read by every later kernel.
