@@ -1,7 +1,7 @@
 """Randomised properties of the oracle (hypothesis): invariants that must hold for any shape,
 kept set and beta, checked on small random layers."""
 import numpy as np
-from hypothesis import given, settings, strategies as st
+from hypothesis import example, given, settings, strategies as st
 
 from oracle import moe_oracle as O
 from paper_2402_14800_b200 import synth
@@ -17,7 +17,7 @@ def layer(h, f, E, T, seed):
 masks = st.integers(min_value=0, max_value=255).filter(lambda m: bin(m).count("1") >= 2)
 
 
-@settings(max_examples=25, deadline=None)
+@settings(max_examples=25, deadline=None, derandomize=True)
 @given(seed=st.integers(0, 10_000), kept=masks, beta=st.floats(0.0, 1.5))
 def test_forward_invariants(seed, kept, beta):
     c = layer(64, 64, 8, 24, seed)
@@ -29,36 +29,49 @@ def test_forward_invariants(seed, kept, beta):
     assert (o["wn"][:, 0] >= o["wn"][:, 1]).all() and (o["wn"] >= 0).all()
     # the skip decision is the strict comparison of the reported ratio with beta
     assert np.array_equal(o["skipped"].astype(bool), o["ratio"] < np.float32(beta))
-    assert ((o["wn"][:, 1] == 0) == o["skipped"].astype(bool)).all()
-    assert (o["ratio"] <= 1.0).all() and (o["ratio"] > 0).all()
+    # a skipped token has no second weight; an unskipped one has none only when exp() underflowed
+    sk = o["skipped"].astype(bool)
+    assert (o["wn"][sk, 1] == 0).all()
+    assert (o["ratio"][~sk & (o["wn"][:, 1] == 0)] < 1e-37).all()
+    assert (o["ratio"] <= 1.0).all() and (o["ratio"] >= 0).all()
     # raising beta can only skip more tokens; the kept routing is untouched by beta
     o2 = O.moe_forward(c["x"], c["Wg"], c["W1"], c["W3"], c["W2"], kept, beta + 0.25)
     assert (o2["skipped"] >= o["skipped"]).all() and np.array_equal(o2["idx"], o["idx"])
 
 
-@settings(max_examples=10, deadline=None)
+@settings(max_examples=10, deadline=None, derandomize=True)
 @given(seed=st.integers(0, 10_000), r=st.integers(2, 8))
+@example(seed=490, r=2)     # a disturbed token whose second weight (4e-24) leaves no trace in the sum
 def test_search_invariants(seed, r):
     c = layer(64, 64, 8, 20, seed)
     s = O.prune_search_allexperts(c["x"], c["Wg"], c["W1"], c["W3"], c["W2"], r)
-    idx = O.route(c["x"], c["Wg"], 0xFF, 0.0)["idx"]
+    rt = O.route(c["x"], c["Wg"], 0xFF, 0.0)
+    idx = rt["idx"]
     pair = (1 << idx[:, 0]) | (1 << idx[:, 1])
+    # A token is disturbed when one of its two experts is pruned.  Its error is non-zero unless
+    # only the second expert went and that expert's weight was below double rounding of the sum
+    # (any replacement weighs even less), so the count lies between the two routing-only counts.
+    faint = rt["wn"][:, 1] < 1e-12
+    slack = 0
     for C, n, loss in zip(s["subsets"], s["n_changed"], s["losses"]):
         assert bin(int(C)).count("1") == r
-        assert n == int(((pair & ~int(C)) != 0).sum())
+        disturbed = (pair & ~int(C)) != 0
+        lost_first = ((1 << idx[:, 0]) & ~int(C)) != 0
+        assert int((disturbed & (lost_first | ~faint)).sum()) <= n <= int(disturbed.sum())
+        slack = max(slack, int((disturbed & ~lost_first & faint).sum()))
         assert (loss == 0.0) == (n == 0)
     assert s["best_subset"] == int(s["subsets"][int(np.argmin(s["losses"]))])
-    # a superset of experts never disturbs more tokens than its subset
+    # a superset of experts never disturbs more tokens than its subset (up to the faint ones)
     if r < 8:
         big = O.prune_search_allexperts(c["x"], c["Wg"], c["W1"], c["W3"], c["W2"], r + 1)
         lookup = {int(C): n for C, n in zip(big["subsets"], big["n_changed"])}
         for C, n in zip(s["subsets"], s["n_changed"]):
             for e in range(8):
                 if not (int(C) >> e) & 1:
-                    assert lookup[int(C) | (1 << e)] <= n
+                    assert lookup[int(C) | (1 << e)] <= n + slack
 
 
-@settings(max_examples=15, deadline=None)
+@settings(max_examples=15, deadline=None, derandomize=True)
 @given(seed=st.integers(0, 10_000), k=st.integers(1, 6), beta=st.floats(0.0, 1.0))
 def test_topk_invariants(seed, k, beta):
     c = layer(64, 64, 8, 16, seed)
@@ -68,6 +81,6 @@ def test_topk_invariants(seed, k, beta):
         assert len(set(o["idx"][t].tolist())) == k
         l = o["logits"][t][o["idx"][t]]
         assert (np.diff(l) <= 0).all()                      # decreasing routing weight
-        assert (o["wn"][t, o["n_active"][t]:] == 0).all() and (o["wn"][t, :o["n_active"][t]] > 0).all()
+        assert (o["wn"][t, o["n_active"][t]:] == 0).all() and (o["wn"][t, :o["n_active"][t]] >= 0).all()
     np.testing.assert_allclose(o["wn"].sum(1), 1.0, rtol=1e-6)
     assert (o["tail_frac"] <= beta + 1e-6).all()
