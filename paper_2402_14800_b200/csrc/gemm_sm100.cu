@@ -1120,6 +1120,11 @@ simt_down_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W2, GemmAr
 
 // ------------------------------------------------------------------------- tensor maps
 
+// L2 promotion size of every tensor map (a build-time knob for side-by-side measurements).
+#ifndef MOE_L2_PROMOTION
+#define MOE_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_256B
+#endif
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -1148,7 +1153,7 @@ int make_map_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows,
   cuuint32_t es[2] = {1, 1};
   CUresult rc = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
                          strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_SWIZZLE_128B, MOE_L2_PROMOTION,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? 0 : -(int)rc;
 }
@@ -1162,7 +1167,7 @@ int make_map_3d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows,
   cuuint32_t es[3] = {1, 1, 1};
   CUresult rc = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims,
                          strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_SWIZZLE_128B, MOE_L2_PROMOTION,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? 0 : -(int)rc;
 }
