@@ -183,7 +183,10 @@ int ensure_gemm(moe_layer* L, int T, int k = 2) {
   if ((rc = grow(L, L->ws->xperm, (size_t)need * L->h * 2))) return rc;
   if ((rc = grow(L, L->ws->act, (size_t)need * L->f * 2))) return rc;
   if ((rc = grow(L, L->ws->O, need_O * 4))) return rc;
+  const void* tail_before = L->ws->tail.p;
   if ((rc = grow(L, L->ws->tail, kTailBufferBytes))) return rc;
+  if (L->ws->tail.p != tail_before)  // the arrival counters start at zero and return to zero
+    CUDA_TRY(cudaMemsetAsync(L->ws->tail.p, 0, kTailHeaderBytes, L->stream));
   L->ws->cap_rows = need;
   L->ws->map_h = L->h;
   L->ws->map_f = L->f;
@@ -305,6 +308,7 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   if (wm) {
     gu.tail = (float*)L->ws->tail.p; dn.tail = (float*)L->ws->tail.p;
     gu.tail_info = (int*)L->ws->status.p + 1; dn.tail_info = (int*)L->ws->status.p + 1;
+    gu.tail_fold = dn.tail_fold = T <= kFoldMaxTokens;
   }
   const int ksplit = wm ? ksplit_for(L) : 1;
   const size_t split_stride = (size_t)rows_cap * L->h;
@@ -523,6 +527,7 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
   if (wm) {
     gu.tail = (float*)W.tail.p; dn.tail = (float*)W.tail.p;
     gu.tail_info = (int*)W.status.p + 1; dn.tail_info = (int*)W.status.p + 1;
+    gu.tail_fold = dn.tail_fold = T <= kFoldMaxTokens;
   }
   const int ksplit = wm ? ksplit_for(L) : 1;
   const size_t split_stride = (size_t)rows_cap * L->h;

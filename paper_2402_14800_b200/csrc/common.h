@@ -167,11 +167,18 @@ struct GemmArgs {
   void* out;               // bf16 activations / fp32 outputs / bf16 expert outputs
   long long split_stride;  // elements between split-K partial planes (decode down-proj)
   int* status;             // device error word
-  float* tail;             // weight-major kernel: partial tiles of K-sliced tail items, or null
+  // weight-major kernel: arrival counters (kTailHeaderBytes, zero between launches) followed by
+  // the partial tiles of the K-sliced tail items; null = no slicing
+  float* tail;
   int* tail_info;          // [0] = number of K-sliced tail items of the launch before a fix-up
+  // 1: no expert holds more than kFoldMaxTokens tokens, the slice of a tail item that finishes
+  // last folds it inside the kernel and no fix-up launch follows
+  int tail_fold;
 };
 
-constexpr size_t kTailBufferBytes = (size_t)256 * 128 * 128 * 4;  // one 64 KB slot per CTA
+constexpr int kFoldMaxTokens = 16;
+constexpr size_t kTailHeaderBytes = 4096;  // four arrival counters per tail item
+constexpr size_t kTailBufferBytes = kTailHeaderBytes + (size_t)256 * 128 * 128 * 4;  // 256 slots of 128 tokens
 
 int gemm_init_driver_api();  // resolves cuTensorMapEncodeTiled; 0 on success
 int make_map_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows);

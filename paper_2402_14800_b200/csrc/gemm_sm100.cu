@@ -752,18 +752,37 @@ constexpr int WM_BN = 128;
 struct ItemW {
   int c, mt, ks, tok_row, out_row, cnt, bucket, kb0, kb1;
   int tail_slot;  // >= 0: this is one K-slice of a tail item and goes to the tail buffer
+  int tail_item;  // which tail item the slice belongs to
+  int nslice;     // non-empty K-slices of that tail item
 };
 
 // Work list of the weight-major kernel.  The base items (expert row tile x weight tile x
-// k-chunk) are dealt round-robin to the `grid` CTAs.  When the last round would be less than
-// half full, its `rem` items are cut into `KSt` K-slices each, so that the last round costs
-// 1/KSt of an item instead of a whole one; the slices leave fp32 partial tiles in the tail
-// buffer and tail_fixup_kernel folds them into the regular output.
+// k-chunk) are dealt round-robin to the `grid` CTAs.  The `rem` items left over after the full
+// rounds would keep part of the machine busy for a whole item's time, so they can be cut into
+// `KSt` K-slices each, dealt like items; the slices leave fp32 partial tiles in the tail buffer
+// and are added up in slice order afterwards.  Two regimes:
+//  * batches of at most kFoldMaxTokens tokens per expert (args.tail_fold): any remainder may be
+//    sliced; KSt minimises the modelled time of the tail, rounds x (k-blocks per slice +
+//    kSliceFixedKb), among the values whose slices fit the buffer (KSt = 1, no slicing, competes
+//    too); the slice that finishes last folds the item inside the kernel.
+//  * larger batches: a remainder of at most half a round is sliced so that one round of slices
+//    fills the machine; tail_fixup_kernel folds the items in a launch of its own.
 struct SchedW {
   int Mt, KS, KB, kb_per_item;
   int n_base, full, rem, KSt, kbs, n_total;
+  int slot_floats;  // floats between the partial tiles of two slices
 };
 
+#ifndef MOE_SLICE_FIXED_KB
+#define MOE_SLICE_FIXED_KB 6
+#endif
+constexpr int kMinSliceKb = 4;                     // a slice covers at least this many k-blocks
+constexpr int kSliceFixedKb = MOE_SLICE_FIXED_KB;  // modelled fixed cost of a slice, in k-blocks
+constexpr int kFoldSlotFloats = 128 * kFoldMaxTokens;
+constexpr int kTailSlotFloats = 128 * WM_BN;  // one partial tile: [token][weight row] fp32
+constexpr int kTailHeaderFloats = (int)(kTailHeaderBytes / 4);  // arrival counters come first
+
+// With args.tail_fold set this is warp-collective: all 32 lanes of a converged warp call it.
 __device__ __forceinline__ SchedW make_sched_w(const Meta& m, const GemmArgs& a, int kb_per_item,
                                                int grid) {
   SchedW s;
@@ -776,15 +795,31 @@ __device__ __forceinline__ SchedW make_sched_w(const Meta& m, const GemmArgs& a,
   s.rem = s.n_base - s.full;
   s.KSt = 1;
   s.kbs = kb_per_item;
-  if (a.tail != nullptr && s.rem > 0 && 2 * s.rem <= grid) {
-    int kst = grid / s.rem;
-    const int cap = kb_per_item / 4 > 1 ? kb_per_item / 4 : 1;  // slices of at least 4 k-blocks
-    if (kst > cap) kst = cap;
-    s.kbs = (kb_per_item + kst - 1) / kst;
-    s.KSt = (kb_per_item + s.kbs - 1) / s.kbs;
+  s.slot_floats = a.tail_fold ? kFoldSlotFloats : kTailSlotFloats;
+  if (a.tail != nullptr && s.rem > 0) {
+    if (a.tail_fold) {
+      const int n_slots = (int)((kTailBufferBytes - kTailHeaderBytes) / ((size_t)kFoldSlotFloats * 4));
+      const int want = (int)(threadIdx.x & 31) + 1;  // this lane tries `want` slices per item
+      const int kbs = (kb_per_item + want - 1) / want;
+      const int kst = (kb_per_item + kbs - 1) / kbs;
+      const int slices = s.rem * kst;
+      const bool valid = want == 1 || (kbs >= kMinSliceKb && slices <= n_slots);
+      const int rounds = (slices + grid - 1) / grid;
+      const unsigned cost = valid ? (unsigned)(rounds * (kbs + kSliceFixedKb)) : 0xffffffu;
+      const unsigned best = __reduce_min_sync(0xffffffffu, (cost << 6) | (unsigned)kst);
+      s.KSt = (int)(best & 63u);
+      s.kbs = (kb_per_item + s.KSt - 1) / s.KSt;
+    } else if (2 * s.rem <= grid) {
+      int kst = grid / s.rem;
+      const int cap = kb_per_item / kMinSliceKb > 1 ? kb_per_item / kMinSliceKb : 1;
+      if (kst > cap) kst = cap;
+      s.kbs = (kb_per_item + kst - 1) / kst;
+      s.KSt = (kb_per_item + s.kbs - 1) / s.kbs;
+    }
   }
   if (s.KSt <= 1) {
     s.KSt = 1;
+    s.kbs = kb_per_item;
     s.full = s.n_base;
     s.rem = 0;
   }
@@ -819,13 +854,55 @@ __device__ __forceinline__ void decode_item_w(const Meta& m, const GemmArgs& a, 
   w.kb0 = ks * s.kb_per_item;
   w.kb1 = min(s.KB, w.kb0 + s.kb_per_item);
   if (w.tail_slot >= 0) {
+    w.tail_item = w.tail_slot / s.KSt;
+    w.nslice = (w.kb1 - w.kb0 + s.kbs - 1) / s.kbs;  // a short last k-chunk has fewer slices
     w.kb0 += sub * s.kbs;
-    w.kb1 = min(w.kb1, w.kb0 + s.kbs);  // may be empty for a short last k-chunk
+    w.kb1 = min(w.kb1, w.kb0 + s.kbs);  // empty beyond nslice
   }
 }
 
-constexpr int kTailSlotFloats = 128 * WM_BN;  // one partial tile: [token][weight row] fp32
 constexpr int kFixupTokens = 2;  // tokens of a tail tile folded by one fix-up block
+
+// Adds up the K-slices of one tail item for the 32 weight rows of epilogue warp `wq` (this
+// lane: one weight row, NT >= w.cnt tokens) in slice order and writes the regular output.
+// SUB slices are loaded before they are added, so that NT x SUB loads are in flight.
+template <bool GATE_UP, int NT, int SUB>
+__device__ __forceinline__ void fold_slices(const GemmArgs& args, const ItemW& w, const float* src,
+                                            int wq, int lane) {
+  float acc[NT];
+#pragma unroll
+  for (int i = 0; i < NT; ++i) acc[i] = 0.f;
+  for (int sub0 = 0; sub0 < w.nslice; sub0 += SUB) {
+    float v[SUB][NT];
+#pragma unroll
+    for (int u = 0; u < SUB; ++u)
+#pragma unroll
+      for (int i = 0; i < NT; ++i)
+        v[u][i] = (sub0 + u < w.nslice && i < w.cnt)
+                      ? __ldcg(src + (size_t)(sub0 + u) * kFoldSlotFloats + i * 128) : 0.f;
+#pragma unroll
+    for (int u = 0; u < SUB; ++u)
+#pragma unroll
+      for (int i = 0; i < NT; ++i) acc[i] += v[u][i];
+  }
+  const int wrow = w.mt * 128 + 32 * wq + lane;
+  const int feat = (wrow >> 5) * kInterleave + (lane & 15);
+  const bool rows_ok = w.mt * 128 + 32 * wq < args.n_w_rows;
+#pragma unroll
+  for (int i = 0; i < NT; ++i) {
+    if (i < w.cnt) {
+      if (GATE_UP) {
+        const float other = __shfl_xor_sync(0xffffffffu, acc[i], 16);
+        if (rows_ok && lane < 16)
+          reinterpret_cast<bf16*>(args.out)[(long long)(w.out_row + i) * args.out_ld + feat] =
+              __float2bfloat16_rn(silu_mul(acc[i], other));
+      } else if (wrow < args.n_w_rows) {
+        reinterpret_cast<float*>(args.out)[(long long)w.ks * args.split_stride +
+                                           (long long)(w.out_row + i) * args.out_ld + wrow] = acc[i];
+      }
+    }
+  }
+}
 
 template <bool GATE_UP>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -855,7 +932,7 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   const int n_items = sched.n_total;
   uint32_t issued = 0;
   // the fix-up launch that follows only needs `rem` blocks: tell it, so the others leave at once
-  if (blockIdx.x == 0 && threadIdx.x == 0 && args.tail_info) args.tail_info[0] = sched.rem;
+  if (blockIdx.x == 0 && threadIdx.x == 0 && args.tail_info && !args.tail_fold) args.tail_info[0] = sched.rem;
 
   if (warp == 0) {
     uint32_t it = 0;
@@ -938,7 +1015,8 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
       const int nchunk = (w.cnt + 15) >> 4;
       if (w.tail_slot >= 0) {
         // K-slice of a tail item: raw fp32 partial tile [token][weight row of the tile]
-        float* outp = args.tail + (size_t)w.tail_slot * kTailSlotFloats + 32 * wq + lane;
+        float* slots = args.tail + kTailHeaderFloats;
+        float* outp = slots + (size_t)w.tail_slot * sched.slot_floats + 32 * wq + lane;
 #pragma unroll 1
         for (int j = 0; j < nchunk; ++j) {
           uint32_t v[16];
@@ -949,6 +1027,32 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
             const int n = 16 * j + i;
             if (n < w.cnt) outp[n * 128] = __uint_as_float(v[i]);
           }
+        }
+        if (args.tail_fold) {
+          // The accumulator has been read: hand the buffer back before the slower part.  Each
+          // epilogue warp owns 32 weight rows of the tile in every slice; it counts its arrival,
+          // and the warp that arrives last adds the slices up in slice order and writes the
+          // regular output, so the order of arrival does not change the result.
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[buf]));
+          ++tile_it;
+          __threadfence();
+          __syncwarp();
+          int* counter = reinterpret_cast<int*>(args.tail) + w.tail_item * 4 + wq;
+          int last = 0;
+          if (lane == 0) last = atomicAdd(counter, 1) == w.nslice - 1;
+          last = __shfl_sync(0xffffffffu, last, 0);
+          if (!last) continue;
+          __threadfence();
+          const float* src = slots + (size_t)(w.tail_item * sched.KSt) * kFoldSlotFloats + 32 * wq + lane;
+          // few tokens: many slices in flight per token; many tokens: many tokens in flight
+          if (w.cnt <= 2) fold_slices<GATE_UP, 2, 16>(args, w, src, wq, lane);
+          else if (w.cnt <= 4) fold_slices<GATE_UP, 4, 8>(args, w, src, wq, lane);
+          else if (w.cnt <= 8) fold_slices<GATE_UP, 8, 4>(args, w, src, wq, lane);
+          else fold_slices<GATE_UP, kFoldMaxTokens, 2>(args, w, src, wq, lane);
+          if (lane == 0) *counter = 0;  // ready for the next launch
+          continue;
         }
       } else if (GATE_UP) {
         // lanes 0-15 hold gate rows, lanes 16-31 the up rows of the same 16 features
@@ -1026,7 +1130,7 @@ tail_fixup_kernel(const GemmArgs args, int kb_per_item, int gemm_grid) {
   __syncthreads();
   const ItemW w = s_w;
   const int nslice = s_nslice;
-  const float* slot0 = args.tail + (size_t)(blockIdx.x * s_kst) * kTailSlotFloats;
+  const float* slot0 = args.tail + kTailHeaderFloats + (size_t)(blockIdx.x * s_kst) * kTailSlotFloats;
   // blockIdx.y walks the tokens of the tile in groups of kFixupTokens; every output is the sum
   // of nslice independent loads
   const int n_begin = blockIdx.y * kFixupTokens;
@@ -1241,12 +1345,12 @@ cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const Gemm
   if (gate_up) {
     cudaError_t e = launch_pdl(gemm_weights_m_kernel<true>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
                                kb_per_item);
-    if (e != cudaSuccess || !a.tail) return e;
+    if (e != cudaSuccess || !a.tail || a.tail_fold) return e;
     return launch_pdl(tail_fixup_kernel<true>, dim3(grid / 2, (mt + kFixupTokens - 1) / kFixupTokens), dim3(128), 0, st, a, kb_per_item, grid);
   }
   cudaError_t e = launch_pdl(gemm_weights_m_kernel<false>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
                              kb_per_item);
-  if (e != cudaSuccess || !a.tail) return e;
+  if (e != cudaSuccess || !a.tail || a.tail_fold) return e;
   return launch_pdl(tail_fixup_kernel<false>, dim3(grid / 2, (mt + kFixupTokens - 1) / kFixupTokens), dim3(128), 0, st, a, kb_per_item, grid);
 }
 
