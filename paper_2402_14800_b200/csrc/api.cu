@@ -216,6 +216,8 @@ int check_status(moe_layer* L) {
   CUDA_TRY(cudaStreamSynchronize(L->stream));
   if (st != 0) {
     cudaMemsetAsync(L->ws->status.p, 0, 4, L->stream);
+    // an aborted GEMM may have left arrival counters of its K-sliced tail items behind
+    if (L->ws->tail.p) cudaMemsetAsync(L->ws->tail.p, 0, kTailHeaderBytes, L->stream);
     return fail(MOE_ERR_DEVICE_TIMEOUT, "a bounded wait inside a GEMM kernel expired");
   }
   return MOE_OK;
