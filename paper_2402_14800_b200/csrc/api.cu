@@ -226,7 +226,7 @@ int check_status(moe_layer* L) {
 // The two grouped GEMMs of the experts over a batch described by `meta`.
 int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmMaps& m_gu,
                      const GemmMaps& m_dn, GemmArgs gu, GemmArgs dn, GemmOut dn_kind,
-                     const bf16* gu_A, const bf16* dn_A, int simt_rows, int max_tokens = 128) {
+                     const bf16* gu_A, const bf16* dn_A, int simt_rows) {
   gu.meta = meta; dn.meta = meta;
   gu.r = L->r; dn.r = L->r;
   gu.K = L->h; gu.n_w_rows = 2 * L->f;
@@ -237,9 +237,9 @@ int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmM
     mark(L);
     CUDA_TRY(launch_simt_down(dn_A, L->W2, dn, simt_rows, dn_kind, L->stream));
   } else if (weights_m) {
-    CUDA_TRY(launch_gemm_weights_m(true, m_gu, gu, (L->h + 63) / 64, max_tokens, L->stream));
+    CUDA_TRY(launch_gemm_weights_m(true, m_gu, gu, (L->h + 63) / 64, L->stream));
     mark(L);
-    CUDA_TRY(launch_gemm_weights_m(false, m_dn, dn, kDecodeKbPerItem, max_tokens, L->stream));
+    CUDA_TRY(launch_gemm_weights_m(false, m_dn, dn, kDecodeKbPerItem, L->stream));
   } else {
     CUDA_TRY(launch_gemm_tokens_m(true, kOutActBf16, m_gu, gu, L->stream));
     mark(L);
@@ -309,8 +309,6 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   const bool wm = dec && !L->debug_simt;
   if (wm) {
     gu.tail = (float*)L->ws->tail.p; dn.tail = (float*)L->ws->tail.p;
-    gu.tail_info = (int*)L->ws->status.p + 1; dn.tail_info = (int*)L->ws->status.p + 1;
-    gu.tail_fold = dn.tail_fold = T <= kFoldMaxTokens;
   }
   const int ksplit = wm ? ksplit_for(L) : 1;
   const size_t split_stride = (size_t)rows_cap * L->h;
@@ -321,7 +319,7 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   memcpy(m_gu.t, L->ws->tok_x, sizeof(m_gu.t));
   memcpy(m_dn.t, L->ws->tok_act, sizeof(m_dn.t));
   rc = run_expert_gemms(L, meta, wm, m_gu, m_dn, gu, dn, kOutF32, (const bf16*)L->ws->xperm.p,
-                        (const bf16*)L->ws->act.p, rows_cap, T);
+                        (const bf16*)L->ws->act.p, rows_cap);
   if (rc) return rc;
   mark(L);
   if (dist)
@@ -528,8 +526,6 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
   const bool wm = dec && !L->debug_simt;
   if (wm) {
     gu.tail = (float*)W.tail.p; dn.tail = (float*)W.tail.p;
-    gu.tail_info = (int*)W.status.p + 1; dn.tail_info = (int*)W.status.p + 1;
-    gu.tail_fold = dn.tail_fold = T <= kFoldMaxTokens;
   }
   const int ksplit = wm ? ksplit_for(L) : 1;
   const size_t split_stride = (size_t)rows_cap * L->h;
@@ -542,7 +538,7 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
   const bool prof_saved = L->prof;
   L->prof = false;
   rc = run_expert_gemms(L, meta, wm, m_gu, m_dn, gu, dn, kOutF32, (const bf16*)W.xperm.p,
-                        (const bf16*)W.act.p, rows_cap, T);
+                        (const bf16*)W.act.p, rows_cap);
   L->prof = prof_saved;
   if (rc) return rc;
   CUDA_TRY(launch_combine_topk((const float*)W.O.p, ksplit, split_stride, (int32_t*)W.k_pos.p,

@@ -170,15 +170,10 @@ struct GemmArgs {
   // weight-major kernel: arrival counters (kTailHeaderBytes, zero between launches) followed by
   // the partial tiles of the K-sliced tail items; null = no slicing
   float* tail;
-  int* tail_info;          // [0] = number of K-sliced tail items of the launch before a fix-up
-  // 1: no expert holds more than kFoldMaxTokens tokens, the slice of a tail item that finishes
-  // last folds it inside the kernel and no fix-up launch follows
-  int tail_fold;
 };
 
-constexpr int kFoldMaxTokens = 16;
 constexpr size_t kTailHeaderBytes = 4096;  // four arrival counters per tail item
-constexpr size_t kTailBufferBytes = kTailHeaderBytes + (size_t)256 * 128 * 128 * 4;  // 256 slots of 128 tokens
+constexpr size_t kTailBufferBytes = kTailHeaderBytes + (size_t)1024 * 128 * 128 * 4;  // 1024 slots of 128 tokens
 
 int gemm_init_driver_api();  // resolves cuTensorMapEncodeTiled; 0 on success
 int make_map_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows);
@@ -195,7 +190,7 @@ cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps&
                                  const GemmArgs& a, cudaStream_t st);
 // Weight rows are the 128-row MMA operand, tokens the narrow one (small T): weights stream once.
 cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
-                                  int kb_per_item, int max_tokens_per_tile, cudaStream_t st);
+                                  int kb_per_item, cudaStream_t st);
 // Plain CUDA-core kernels of the same contractions, for bring-up and debugging only
 // (MOE_DEBUG_SIMT=1); never selected otherwise.
 cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,

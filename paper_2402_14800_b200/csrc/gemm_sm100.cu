@@ -758,31 +758,33 @@ struct ItemW {
 
 // Work list of the weight-major kernel.  The base items (expert row tile x weight tile x
 // k-chunk) are dealt round-robin to the `grid` CTAs.  The `rem` items left over after the full
-// rounds would keep part of the machine busy for a whole item's time, so they can be cut into
-// `KSt` K-slices each, dealt like items; the slices leave fp32 partial tiles in the tail buffer
-// and are added up in slice order afterwards.  Two regimes:
-//  * batches of at most kFoldMaxTokens tokens per expert (args.tail_fold): any remainder may be
-//    sliced; KSt minimises the modelled time of the tail, rounds x (k-blocks per slice +
-//    kSliceFixedKb), among the values whose slices fit the buffer (KSt = 1, no slicing, competes
-//    too); the slice that finishes last folds the item inside the kernel.
-//  * larger batches: a remainder of at most half a round is sliced so that one round of slices
-//    fills the machine; tail_fixup_kernel folds the items in a launch of its own.
+// rounds would keep part of the machine busy for a whole item's time, so they are cut into
+// `KSt` K-slices each.  The slices come FIRST in the work list and are dealt like items; each
+// leaves an fp32 partial tile in the tail buffer, and the slice of an item that finishes last
+// adds the partial tiles up in slice order and writes the regular output (the order of arrival
+// does not change the result).  That happens while the CTAs are busy with their regular items,
+// off the critical path, and the last round of the launch is a full one.
+// KSt minimises the modelled time of the slices, rounds x (k-blocks per slice + kSliceFixedKb),
+// among the values whose slices fit the tail buffer and whose fold stays below kFoldLoads loads
+// per thread; KSt = 1 (no slicing) competes too.
 struct SchedW {
   int Mt, KS, KB, kb_per_item;
-  int n_base, full, rem, KSt, kbs, n_total;
+  int n_base, full, rem, KSt, kbs, n_slices, n_total;
   int slot_floats;  // floats between the partial tiles of two slices
 };
 
 #ifndef MOE_SLICE_FIXED_KB
 #define MOE_SLICE_FIXED_KB 6
 #endif
+#ifndef MOE_FOLD_LOADS
+#define MOE_FOLD_LOADS 512
+#endif
 constexpr int kMinSliceKb = 4;                     // a slice covers at least this many k-blocks
 constexpr int kSliceFixedKb = MOE_SLICE_FIXED_KB;  // modelled fixed cost of a slice, in k-blocks
-constexpr int kFoldSlotFloats = 128 * kFoldMaxTokens;
-constexpr int kTailSlotFloats = 128 * WM_BN;  // one partial tile: [token][weight row] fp32
+constexpr int kFoldLoads = MOE_FOLD_LOADS;         // tokens x slices one thread adds up at most
 constexpr int kTailHeaderFloats = (int)(kTailHeaderBytes / 4);  // arrival counters come first
 
-// With args.tail_fold set this is warp-collective: all 32 lanes of a converged warp call it.
+// Warp-collective: all 32 lanes of a converged warp call it and get the same result.
 __device__ __forceinline__ SchedW make_sched_w(const Meta& m, const GemmArgs& a, int kb_per_item,
                                                int grid) {
   SchedW s;
@@ -795,27 +797,23 @@ __device__ __forceinline__ SchedW make_sched_w(const Meta& m, const GemmArgs& a,
   s.rem = s.n_base - s.full;
   s.KSt = 1;
   s.kbs = kb_per_item;
-  s.slot_floats = a.tail_fold ? kFoldSlotFloats : kTailSlotFloats;
+  int maxcnt = 1;
+  for (int c = 0; c < a.r; ++c) maxcnt = max(maxcnt, min(m.count[c], WM_BN));
+  const int slot_tokens = (maxcnt + 15) & ~15;
+  s.slot_floats = 128 * slot_tokens;
   if (a.tail != nullptr && s.rem > 0) {
-    if (a.tail_fold) {
-      const int n_slots = (int)((kTailBufferBytes - kTailHeaderBytes) / ((size_t)kFoldSlotFloats * 4));
-      const int want = (int)(threadIdx.x & 31) + 1;  // this lane tries `want` slices per item
-      const int kbs = (kb_per_item + want - 1) / want;
-      const int kst = (kb_per_item + kbs - 1) / kbs;
-      const int slices = s.rem * kst;
-      const bool valid = want == 1 || (kbs >= kMinSliceKb && slices <= n_slots);
-      const int rounds = (slices + grid - 1) / grid;
-      const unsigned cost = valid ? (unsigned)(rounds * (kbs + kSliceFixedKb)) : 0xffffffu;
-      const unsigned best = __reduce_min_sync(0xffffffffu, (cost << 6) | (unsigned)kst);
-      s.KSt = (int)(best & 63u);
-      s.kbs = (kb_per_item + s.KSt - 1) / s.KSt;
-    } else if (2 * s.rem <= grid) {
-      int kst = grid / s.rem;
-      const int cap = kb_per_item / kMinSliceKb > 1 ? kb_per_item / kMinSliceKb : 1;
-      if (kst > cap) kst = cap;
-      s.kbs = (kb_per_item + kst - 1) / kst;
-      s.KSt = (kb_per_item + s.kbs - 1) / s.kbs;
-    }
+    const int n_slots = (int)((kTailBufferBytes - kTailHeaderBytes) / ((size_t)s.slot_floats * 4));
+    const int kst_fold = kFoldLoads / slot_tokens;
+    const int want = (int)(threadIdx.x & 31) + 1;  // this lane tries `want` slices per item
+    const int kbs = (kb_per_item + want - 1) / want;
+    const int kst = (kb_per_item + kbs - 1) / kbs;
+    const int slices = s.rem * kst;
+    const bool valid = want == 1 || (kbs >= kMinSliceKb && slices <= n_slots && kst <= kst_fold);
+    const int rounds = (slices + grid - 1) / grid;
+    const unsigned cost = valid ? (unsigned)(rounds * (kbs + kSliceFixedKb)) : 0xffffffu;
+    const unsigned best = __reduce_min_sync(0xffffffffu, (cost << 6) | (unsigned)kst);
+    s.KSt = (int)(best & 63u);
+    s.kbs = (kb_per_item + s.KSt - 1) / s.KSt;
   }
   if (s.KSt <= 1) {
     s.KSt = 1;
@@ -823,19 +821,19 @@ __device__ __forceinline__ SchedW make_sched_w(const Meta& m, const GemmArgs& a,
     s.full = s.n_base;
     s.rem = 0;
   }
-  s.n_total = s.full + s.rem * s.KSt;
+  s.n_slices = s.rem * s.KSt;
+  s.n_total = s.n_slices + s.full;
   return s;
 }
 
 __device__ __forceinline__ void decode_item_w(const Meta& m, const GemmArgs& a, const SchedW& s,
                                               int item, ItemW& w) {
-  int base = item, sub = 0;
+  int base = item - s.n_slices, sub = 0;
   w.tail_slot = -1;
-  if (item >= s.full) {
-    const int j = item - s.full;
-    base = s.full + j / s.KSt;
-    sub = j - (j / s.KSt) * s.KSt;
-    w.tail_slot = j;
+  if (item < s.n_slices) {  // the slices come first
+    base = s.full + item / s.KSt;
+    sub = item - (item / s.KSt) * s.KSt;
+    w.tail_slot = item;
   }
   const int ks = base % s.KS;
   const int rest = base / s.KS;
@@ -861,25 +859,24 @@ __device__ __forceinline__ void decode_item_w(const Meta& m, const GemmArgs& a, 
   }
 }
 
-constexpr int kFixupTokens = 2;  // tokens of a tail tile folded by one fix-up block
-
 // Adds up the K-slices of one tail item for the 32 weight rows of epilogue warp `wq` (this
-// lane: one weight row, NT >= w.cnt tokens) in slice order and writes the regular output.
-// SUB slices are loaded before they are added, so that NT x SUB loads are in flight.
+// lane: one weight row) and tokens n0 .. n0 + nt - 1 (nt <= NT) in slice order and writes the
+// regular output.  SUB slices are loaded before they are added: NT x SUB loads are in flight.
 template <bool GATE_UP, int NT, int SUB>
 __device__ __forceinline__ void fold_slices(const GemmArgs& args, const ItemW& w, const float* src,
-                                            int wq, int lane) {
+                                            int slot_floats, int n0, int nt, int wq, int lane) {
   float acc[NT];
 #pragma unroll
   for (int i = 0; i < NT; ++i) acc[i] = 0.f;
+  src += n0 * 128;
   for (int sub0 = 0; sub0 < w.nslice; sub0 += SUB) {
     float v[SUB][NT];
 #pragma unroll
     for (int u = 0; u < SUB; ++u)
 #pragma unroll
       for (int i = 0; i < NT; ++i)
-        v[u][i] = (sub0 + u < w.nslice && i < w.cnt)
-                      ? __ldcg(src + (size_t)(sub0 + u) * kFoldSlotFloats + i * 128) : 0.f;
+        v[u][i] = (sub0 + u < w.nslice && i < nt)
+                      ? __ldcg(src + (size_t)(sub0 + u) * slot_floats + i * 128) : 0.f;
 #pragma unroll
     for (int u = 0; u < SUB; ++u)
 #pragma unroll
@@ -890,15 +887,15 @@ __device__ __forceinline__ void fold_slices(const GemmArgs& args, const ItemW& w
   const bool rows_ok = w.mt * 128 + 32 * wq < args.n_w_rows;
 #pragma unroll
   for (int i = 0; i < NT; ++i) {
-    if (i < w.cnt) {
+    if (i < nt) {
       if (GATE_UP) {
         const float other = __shfl_xor_sync(0xffffffffu, acc[i], 16);
         if (rows_ok && lane < 16)
-          reinterpret_cast<bf16*>(args.out)[(long long)(w.out_row + i) * args.out_ld + feat] =
+          reinterpret_cast<bf16*>(args.out)[(long long)(w.out_row + n0 + i) * args.out_ld + feat] =
               __float2bfloat16_rn(silu_mul(acc[i], other));
       } else if (wrow < args.n_w_rows) {
         reinterpret_cast<float*>(args.out)[(long long)w.ks * args.split_stride +
-                                           (long long)(w.out_row + i) * args.out_ld + wrow] = acc[i];
+                                           (long long)(w.out_row + n0 + i) * args.out_ld + wrow] = acc[i];
       }
     }
   }
@@ -931,8 +928,6 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   const SchedW sched = make_sched_w(s_meta, args, kb_per_item, (int)gridDim.x);
   const int n_items = sched.n_total;
   uint32_t issued = 0;
-  // the fix-up launch that follows only needs `rem` blocks: tell it, so the others leave at once
-  if (blockIdx.x == 0 && threadIdx.x == 0 && args.tail_info && !args.tail_fold) args.tail_info[0] = sched.rem;
 
   if (warp == 0) {
     uint32_t it = 0;
@@ -1028,32 +1023,32 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
             if (n < w.cnt) outp[n * 128] = __uint_as_float(v[i]);
           }
         }
-        if (args.tail_fold) {
-          // The accumulator has been read: hand the buffer back before the slower part.  Each
-          // epilogue warp owns 32 weight rows of the tile in every slice; it counts its arrival,
-          // and the warp that arrives last adds the slices up in slice order and writes the
-          // regular output, so the order of arrival does not change the result.
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[buf]));
-          ++tile_it;
-          __threadfence();
-          __syncwarp();
-          int* counter = reinterpret_cast<int*>(args.tail) + w.tail_item * 4 + wq;
-          int last = 0;
-          if (lane == 0) last = atomicAdd(counter, 1) == w.nslice - 1;
-          last = __shfl_sync(0xffffffffu, last, 0);
-          if (!last) continue;
-          __threadfence();
-          const float* src = slots + (size_t)(w.tail_item * sched.KSt) * kFoldSlotFloats + 32 * wq + lane;
-          // few tokens: many slices in flight per token; many tokens: many tokens in flight
-          if (w.cnt <= 2) fold_slices<GATE_UP, 2, 16>(args, w, src, wq, lane);
-          else if (w.cnt <= 4) fold_slices<GATE_UP, 4, 8>(args, w, src, wq, lane);
-          else if (w.cnt <= 8) fold_slices<GATE_UP, 8, 4>(args, w, src, wq, lane);
-          else fold_slices<GATE_UP, kFoldMaxTokens, 2>(args, w, src, wq, lane);
-          if (lane == 0) *counter = 0;  // ready for the next launch
-          continue;
-        }
+        // The accumulator has been read: hand the buffer back before the slower part.  Each
+        // epilogue warp owns 32 weight rows of the tile in every slice; it counts its arrival,
+        // and the warp that arrives last folds those rows of the item.
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[buf]));
+        ++tile_it;
+        __threadfence();
+        __syncwarp();
+        int* counter = reinterpret_cast<int*>(args.tail) + w.tail_item * 4 + wq;
+        int last = 0;
+        if (lane == 0) last = atomicAdd(counter, 1) == w.nslice - 1;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (!last) continue;
+        __threadfence();
+        const float* src = slots + (size_t)(w.tail_item * sched.KSt) * sched.slot_floats + 32 * wq + lane;
+        const int sf = sched.slot_floats;
+        // few tokens: many slices in flight per token; many tokens: many tokens in flight
+        if (w.cnt <= 2) fold_slices<GATE_UP, 2, 16>(args, w, src, sf, 0, w.cnt, wq, lane);
+        else if (w.cnt <= 4) fold_slices<GATE_UP, 4, 8>(args, w, src, sf, 0, w.cnt, wq, lane);
+        else if (w.cnt <= 8) fold_slices<GATE_UP, 8, 4>(args, w, src, sf, 0, w.cnt, wq, lane);
+        else
+          for (int n0 = 0; n0 < w.cnt; n0 += 16)
+            fold_slices<GATE_UP, 16, 2>(args, w, src, sf, n0, min(16, w.cnt - n0), wq, lane);
+        if (lane == 0) *counter = 0;  // ready for the next launch
+        continue;
       } else if (GATE_UP) {
         // lanes 0-15 hold gate rows, lanes 16-31 the up rows of the same 16 features
         const int feat = (wrow >> 5) * kInterleave + (lane & 15);
@@ -1097,73 +1092,6 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   }
   pdl_launch_dependents();
   teardown<WM_NS, 256>(bars, tmem_base, issued, args.status);
-}
-
-// Folds the K-slices of the tail items into the regular output: the gate/up variant sums the
-// slices and applies silu(g) * u, the down variant sums them into the item's split-K plane.
-template <bool GATE_UP>
-__global__ void __launch_bounds__(128)
-tail_fixup_kernel(const GemmArgs args, int kb_per_item, int gemm_grid) {
-  __shared__ Meta s_meta;
-  __shared__ ItemW s_w;
-  __shared__ int s_nslice, s_kst;
-  pdl_launch_dependents();
-  pdl_wait();
-  if ((int)blockIdx.x >= args.tail_info[0]) return;  // written by the GEMM this launch follows
-  for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
-    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const SchedW sched = make_sched_w(s_meta, args, kb_per_item, gemm_grid);
-    ItemW w;
-    // slices of this tail item, in slice order; empty slices were never written
-    int nslice = 0;
-    for (int sub = 0; sub < sched.KSt; ++sub) {
-      decode_item_w(s_meta, args, sched, sched.full + (int)blockIdx.x * sched.KSt + sub, w);
-      if (w.kb0 < w.kb1) nslice = sub + 1;
-    }
-    decode_item_w(s_meta, args, sched, sched.full + (int)blockIdx.x * sched.KSt, w);
-    s_w = w;
-    s_nslice = nslice;
-    s_kst = sched.KSt;
-  }
-  __syncthreads();
-  const ItemW w = s_w;
-  const int nslice = s_nslice;
-  const float* slot0 = args.tail + kTailHeaderFloats + (size_t)(blockIdx.x * s_kst) * kTailSlotFloats;
-  // blockIdx.y walks the tokens of the tile in groups of kFixupTokens; every output is the sum
-  // of nslice independent loads
-  const int n_begin = blockIdx.y * kFixupTokens;
-  const int n_end = min(w.cnt, n_begin + kFixupTokens);
-  if (GATE_UP) {
-    // 64 features per tile: rows 32q + s are gate, 32q + 16 + s up; two tokens per pass
-    const int fj = threadIdx.x & 63;
-    const int q = fj >> 4, sft = fj & 15;
-    if (w.mt * 128 + 32 * q >= args.n_w_rows) return;
-    const int feat = (w.mt * 4 + q) * kInterleave + sft;
-    for (int n = n_begin + (threadIdx.x >> 6); n < n_end; n += 2) {
-      float g = 0.f, u = 0.f;
-#pragma unroll 8
-      for (int sub = 0; sub < nslice; ++sub) {
-        const float* t = slot0 + (size_t)sub * kTailSlotFloats + n * 128;
-        g += t[32 * q + sft];
-        u += t[32 * q + 16 + sft];
-      }
-      reinterpret_cast<bf16*>(args.out)[(long long)(w.out_row + n) * args.out_ld + feat] =
-          __float2bfloat16_rn(silu_mul(g, u));
-    }
-  } else {
-    const int col = threadIdx.x;
-    const int wrow = w.mt * 128 + col;
-    if (wrow >= args.n_w_rows) return;
-    for (int n = n_begin; n < n_end; ++n) {
-      float v = 0.f;
-#pragma unroll 8
-      for (int sub = 0; sub < nslice; ++sub) v += slot0[(size_t)sub * kTailSlotFloats + n * 128 + col];
-      reinterpret_cast<float*>(args.out)[(long long)w.ks * args.split_stride +
-                                         (long long)(w.out_row + n) * args.out_ld + wrow] = v;
-    }
-  }
 }
 
 // ------------------------------------------------------------ CUDA-core debug kernels
@@ -1339,19 +1267,13 @@ cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps&
 }
 
 cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
-                                  int kb_per_item, int max_tokens_per_tile, cudaStream_t st) {
-  const int mt = max_tokens_per_tile < 1 ? 1 : (max_tokens_per_tile > WM_BN ? WM_BN : max_tokens_per_tile);
+                                  int kb_per_item, cudaStream_t st) {
   const int grid = g_num_sms > 0 ? g_num_sms : 148;
-  if (gate_up) {
-    cudaError_t e = launch_pdl(gemm_weights_m_kernel<true>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
-                               kb_per_item);
-    if (e != cudaSuccess || !a.tail || a.tail_fold) return e;
-    return launch_pdl(tail_fixup_kernel<true>, dim3(grid / 2, (mt + kFixupTokens - 1) / kFixupTokens), dim3(128), 0, st, a, kb_per_item, grid);
-  }
-  cudaError_t e = launch_pdl(gemm_weights_m_kernel<false>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
-                             kb_per_item);
-  if (e != cudaSuccess || !a.tail || a.tail_fold) return e;
-  return launch_pdl(tail_fixup_kernel<false>, dim3(grid / 2, (mt + kFixupTokens - 1) / kFixupTokens), dim3(128), 0, st, a, kb_per_item, grid);
+  if (gate_up)
+    return launch_pdl(gemm_weights_m_kernel<true>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
+                      kb_per_item);
+  return launch_pdl(gemm_weights_m_kernel<false>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
+                    kb_per_item);
 }
 
 cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,
