@@ -14,7 +14,7 @@ typedef __nv_bfloat16 bf16;
 
 constexpr int kMaxE = MOE_MAX_EXPERTS;
 constexpr int kTileRows = 128;            // token rows per row tile of the grouped GEMMs
-constexpr int kRouteTokPerBlock = 64;     // tokens routed by one block (8 warps x 8 tokens)
+constexpr int kRouteTokPerBlock = 16;     // tokens routed by one block (one warp per token)
 constexpr int kHistCols = 2 * kMaxE + 1;  // per (expert, slot) pair counts + skipped count
 constexpr int kInterleave = 16;           // W1/W3 rows are interleaved in groups of 16
 constexpr int kDecodeMaxT = 256;          // up to here the weight-stationary GEMM is used

@@ -223,48 +223,65 @@ permute_gather_small_kernel(const bf16* __restrict__ x, const int32_t* __restric
   }
 }
 
+// Large batches: one warp per token, kRouteTokPerBlock tokens per block (whose pair counts go
+// to the block's histogram row).  A lane first fetches its whole share of the token's row (the
+// loads that come from DRAM, all independent), then walks it against the router rows, which
+// sit in L1 after the block's first pass.
+
 template <int R>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(32 * kRouteTokPerBlock)
 router_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, int h, int r,
               float beta, KeptIds kept, RouteOut o) {
   pdl_launch_dependents();
   pdl_wait();
   __shared__ int s_e[kRouteTokPerBlock][2];
   __shared__ int s_skip[kRouteTokPerBlock];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t0 = blockIdx.x * kRouteTokPerBlock;
+  constexpr int kRouteXVec = R > 8 ? 8 : 16;  // 16-byte vectors of the row a lane holds at a time
+  const int tl = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x * kRouteTokPerBlock + tl;
   const int nvec = h >> 3;
 
-  for (int i = 0; i < kRouteTokPerBlock / 8; ++i) {
-    const int tl = warp * (kRouteTokPerBlock / 8) + i;
-    const int t = t0 + tl;
-    if (t >= T) {
-      if (lane == 0) { s_e[tl][0] = -1; s_e[tl][1] = -1; s_skip[tl] = 0; }
-      continue;
-    }
-    float acc[R];
+  float acc[R];
 #pragma unroll
-    for (int c = 0; c < R; ++c) acc[c] = 0.f;
-    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)t * h);
-    for (int v = lane; v < nvec; v += 32) {
-      float xf[8];
-      unpack8(__ldg(xr + v), xf);
+  for (int c = 0; c < R; ++c) acc[c] = 0.f;
+  // a token past the end reads the last token's row; its result is dropped below
+  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)min(t, T - 1) * h);
+  for (int v0 = lane; v0 < nvec; v0 += 32 * kRouteXVec) {
+    uint4 xv[kRouteXVec];
 #pragma unroll
-      for (int c = 0; c < R; ++c) {
-        if (c < r) {
-          float wf[8];
-          unpack8(__ldg(reinterpret_cast<const uint4*>(Wg + (size_t)c * h) + v), wf);
+    for (int i = 0; i < kRouteXVec; ++i)
+      xv[i] = (v0 + 32 * i < nvec) ? __ldg(xr + v0 + 32 * i) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) acc[c] = fmaf(xf[k], wf[k], acc[c]);
+    for (int i = 0; i < kRouteXVec; ++i) {
+      const int v = v0 + 32 * i;
+      if (v < nvec) {
+        uint4 wv[R];
+#pragma unroll
+        for (int c = 0; c < R; ++c)
+          if (c < r) wv[c] = __ldg(reinterpret_cast<const uint4*>(Wg + (size_t)c * h) + v);
+        float xf[8];
+        unpack8(xv[i], xf);
+#pragma unroll
+        for (int c = 0; c < R; ++c) {
+          if (c < r) {
+            float wf[8];
+            unpack8(wv[c], wf);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc[c] = fmaf(xf[k], wf[k], acc[c]);
+          }
         }
       }
     }
+  }
 #pragma unroll
-    for (int c = 0; c < R; ++c) {
+  for (int c = 0; c < R; ++c) {
 #pragma unroll
-      for (int s = 16; s > 0; s >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], s);
-    }
-    if (lane == 0) {
+    for (int s = 16; s > 0; s >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], s);
+  }
+  if (lane == 0) {
+    if (t >= T) {
+      s_e[tl][0] = -1; s_e[tl][1] = -1; s_skip[tl] = 0;
+    } else {
       int e0, e1;
       bool skip;
       route_decide<R>(acc, r, beta, t, kept, o, e0, e1, skip);
@@ -543,7 +560,7 @@ router_topk_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int 
   if (u_nact) u_nact[t] = istar;
 }
 
-// Per block of 64 tokens: active pairs per expert, in the column layout scan_kernel reads
+// Per block of kRouteTokPerBlock tokens: active pairs per expert, in the column layout scan_kernel reads
 // (the pairs go to the slot-0 column, the skipped pairs to the last column).
 __global__ void __launch_bounds__(kHistCols < 64 ? 64 : kHistCols)
 count_topk_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ nact, int T, int k,
@@ -808,11 +825,11 @@ cudaError_t launch_router(const bf16* x, const bf16* Wg, int T, int h, int r, fl
                           const KeptIds& kept, const RouteOut& out, cudaStream_t st) {
   const int nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
   switch (r) {
-    case 2: return launch_pdl(router_kernel<2>, dim3(nblk), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
-    case 3: case 4: return launch_pdl(router_kernel<4>, dim3(nblk), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
-    case 5: case 6: return launch_pdl(router_kernel<6>, dim3(nblk), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
-    case 7: case 8: return launch_pdl(router_kernel<8>, dim3(nblk), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
-    default: return launch_pdl(router_kernel<kMaxE>, dim3(nblk), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
+    case 2: return launch_pdl(router_kernel<2>, dim3(nblk), dim3(32 * kRouteTokPerBlock), 0, st, x, Wg, T, h, r, beta, kept, out);
+    case 3: case 4: return launch_pdl(router_kernel<4>, dim3(nblk), dim3(32 * kRouteTokPerBlock), 0, st, x, Wg, T, h, r, beta, kept, out);
+    case 5: case 6: return launch_pdl(router_kernel<6>, dim3(nblk), dim3(32 * kRouteTokPerBlock), 0, st, x, Wg, T, h, r, beta, kept, out);
+    case 7: case 8: return launch_pdl(router_kernel<8>, dim3(nblk), dim3(32 * kRouteTokPerBlock), 0, st, x, Wg, T, h, r, beta, kept, out);
+    default: return launch_pdl(router_kernel<kMaxE>, dim3(nblk), dim3(32 * kRouteTokPerBlock), 0, st, x, Wg, T, h, r, beta, kept, out);
   }
   return cudaGetLastError();
 }
