@@ -319,6 +319,8 @@ scan_kernel(const int32_t* __restrict__ blk_hist, int nblk, int r, int pad,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (warp < r) {
     int run = 0, run0 = 0;
+    // the loads of a step do not depend on the running sums: let several steps be in flight
+#pragma unroll 4
     for (int b0 = 0; b0 < nblk; b0 += 32) {
       const int b = b0 + lane;
       int v0 = 0, v1 = 0;
