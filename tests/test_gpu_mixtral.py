@@ -92,16 +92,16 @@ def test_pruned_layers(big, kept, T):
     assert big["layer"](kept).weight_bytes == bin(kept).count("1") * per_expert
 
 
-@pytest.mark.parametrize("T", [1, 3, 16])
+@pytest.mark.parametrize("T", [1, 3, 16, 128, 256])
 def test_small_batches_repeat_bit_for_bit(big, T):
-    # up to 16 tokens the K-slices of the last round are added up inside the GEMM by whichever
+    # the K-slices of the remainder of the work list are added up inside the GEMM by whichever
     # slice finishes last: the result must not depend on the order of arrival
     x = synth.make_tokens(T, H, seed=5, device=DEV)
     for kept in (FULL, 0x3F):
         layer = big["layer"](kept)
         beta = calibrated_beta(big, kept)
         first = layer.forward(x, beta).clone()
-        for _ in range(6):
+        for _ in range(12):
             assert torch.equal(layer.forward(x, beta), first)
 
 
