@@ -296,9 +296,10 @@ def run_ours(a):
     else:
         def step():
             layer.forward(x, beta, y=y)
+        # T = 1: routing (one launch), gate/up GEMM, down GEMM, combine;
         # T <= 256: router, permute+gather, gate/up GEMM, down GEMM, combine;
         # larger T: router, scan, scatter, gather, gate/up GEMM, down GEMM, combine
-        launches_per_step = 5 if a.tokens <= 256 else 7
+        launches_per_step = 4 if a.tokens == 1 else (5 if a.tokens <= 256 else 7)
 
     # routing facts for the algorithmic byte / flop counts (one untimed call)
     pairs = touched = 0
@@ -630,7 +631,7 @@ def run_stack(a):
                     "frac_of_nominal_dense_bf16": ach / NOMINAL_BF16_TFLOPS,
                     "peak_source": peaks["source"] + " (sustained bf16)"}
     if rank == 0:
-        per_layer = (5 if T <= 256 else 7) + 1   # the layer's kernels + its RMSNorm
+        per_layer = (4 if T == 1 else (5 if T <= 256 else 7)) + 1   # the layer's kernels + its RMSNorm
         line = {
             "metric": "MoE-stack tokens/s on 1 B200 (32 layers, RMSNorm + residual, attention omitted)",
             "value": value, "unit": "tokens/s", "n_gpus": world, "steps": a.steps,

@@ -283,7 +283,11 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   Meta* meta = (Meta*)L->ws->meta.p;
   if (L->prof && (L->prof_used % (MOE_PROFILE_STAGES + 1)) != 0) L->prof_used = 0;
   mark(L);
-  if (dec) {
+  if (T == 1) {
+    CUDA_TRY(launch_route_single((const bf16*)x, L->Wg, L->h, L->r, beta, L->kept, ro, 16, meta,
+                                 (int32_t*)L->ws->pair_pos.p, (int32_t*)L->ws->row_token.p,
+                                 (bf16*)L->ws->xperm.p, s_count, s_nsk, s_nt, L->E, st));
+  } else if (dec) {
     CUDA_TRY(launch_router_small((const bf16*)x, L->Wg, T, L->h, L->r, beta, L->kept, ro, st));
     CUDA_TRY(launch_permute_gather_small((const bf16*)x, ro.idx, ro.skipped, T, L->h, L->r, 16, meta,
                                          (int32_t*)L->ws->pair_pos.p, (int32_t*)L->ws->row_token.p,

@@ -108,6 +108,10 @@ cudaError_t launch_router(const bf16* x, const bf16* Wg, int T, int h, int r, fl
 // T <= kDecodeMaxT: router with one block per token; permutation + gather with one block per token
 cudaError_t launch_router_small(const bf16* x, const bf16* Wg, int T, int h, int r, float beta,
                                 const KeptIds& kept, const RouteOut& out, cudaStream_t st);
+cudaError_t launch_route_single(const bf16* x, const bf16* Wg, int h, int r, float beta,
+                                const KeptIds& kept, const RouteOut& out, int pad, Meta* meta,
+                                int32_t* pair_pos, int32_t* row_token, bf16* xperm, int32_t* s_count,
+                                int32_t* s_nskipped, int32_t* s_ntouched, int E, cudaStream_t st);
 cudaError_t launch_permute_gather_small(const bf16* x, const int32_t* idx, const uint8_t* skipped, int T,
                                         int h, int r, int pad, Meta* meta, int32_t* pair_pos,
                                         int32_t* row_token, bf16* xperm, int32_t* s_count,

@@ -120,6 +120,103 @@ router_small_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
   }
 }
 
+// A single token (batch-1 decoding): routing, the (trivial) permutation, the batch description
+// and the copy of the token's row in one block, in place of the two launches above.  The
+// records it writes are those of router_small_kernel + permute_gather_small_kernel for T = 1.
+template <int R>
+__global__ void __launch_bounds__(256)
+route_single_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int h, int r, float beta,
+                    KeptIds kept, RouteOut o, int pad, Meta* meta, int32_t* __restrict__ pair_pos,
+                    int32_t* __restrict__ row_token, bf16* __restrict__ xperm, int32_t* s_count,
+                    int32_t* s_nskipped, int32_t* s_ntouched, int E) {
+  pdl_launch_dependents();
+  pdl_wait();
+  __shared__ float s_part[8][R];
+  __shared__ int s_p[2];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nvec = h >> 3;
+  float acc[R];
+#pragma unroll
+  for (int c = 0; c < R; ++c) acc[c] = 0.f;
+  const uint4* xr = reinterpret_cast<const uint4*>(x);
+  for (int v = threadIdx.x; v < nvec; v += 256) {
+    float xf[8];
+    unpack8(__ldg(xr + v), xf);
+#pragma unroll
+    for (int c = 0; c < R; ++c) {
+      if (c < r) {
+        float wf[8];
+        unpack8(__ldg(reinterpret_cast<const uint4*>(Wg + (size_t)c * h) + v), wf);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[c] = fmaf(xf[k], wf[k], acc[c]);
+      }
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < R; ++c) {
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], s);
+    if (lane == 0) s_part[warp][c] = acc[c];
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float l[R];
+#pragma unroll
+    for (int c = 0; c < R; ++c) {
+      float v = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) v += s_part[w][c];
+      l[c] = v;
+    }
+    int e0, e1;
+    bool skip;
+    route_decide<R>(l, r, beta, 0, kept, o, e0, e1, skip);
+    if (skip) e1 = -1;
+    // the batch description: one row for e0, one for e1 unless it is skipped
+    int off = 0, tiles = 0;
+    meta->off[0] = 0;
+    meta->tile_prefix[0] = 0;
+    for (int c = 0; c < kMaxE; ++c) {
+      const int n0 = (c == e0), n1 = (c == e1);
+      const int n = n0 + n1;
+      if (c == e0) s_p[0] = off;
+      if (c == e1) s_p[1] = off;
+      off += (n + pad - 1) / pad * pad;
+      tiles += (n + kTileRows - 1) / kTileRows;
+      meta->count[c] = n;
+      meta->count_slot[c][0] = n0;
+      meta->count_slot[c][1] = n1;
+      meta->off[c + 1] = off;
+      meta->tile_prefix[c + 1] = tiles;
+    }
+    if (e1 < 0) s_p[1] = -1;
+    meta->rows_total = off;
+    meta->n_skipped = skip ? 1 : 0;
+    meta->n_touched = skip ? 1 : 2;
+    meta->reserved = 0;
+    pair_pos[0] = s_p[0];
+    pair_pos[1] = s_p[1];
+    row_token[s_p[0]] = 0;
+    if (e1 >= 0) row_token[s_p[1]] = 0;
+    if (s_count) {
+      for (int e = 0; e < E; ++e) { s_count[2 * e] = 0; s_count[2 * e + 1] = 0; }
+      s_count[2 * kept.id[e0]] = 1;
+      if (e1 >= 0) s_count[2 * kept.id[e1] + 1] = 1;
+      *s_nskipped = skip ? 1 : 0;
+      *s_ntouched = skip ? 1 : 2;
+    }
+  }
+  __syncthreads();
+  const int p0 = s_p[0], p1 = s_p[1];
+  uint4* d0 = reinterpret_cast<uint4*>(xperm + (size_t)p0 * h);
+  uint4* d1 = reinterpret_cast<uint4*>(xperm + (size_t)(p1 < 0 ? p0 : p1) * h);
+  for (int v = threadIdx.x; v < nvec; v += 256) {
+    const uint4 val = __ldg(xr + v);
+    d0[v] = val;
+    if (p1 >= 0) d1[v] = val;
+  }
+}
+
 // Small batches: permutation and gather in one launch, one block per token.  Every block
 // recomputes the (tiny) histogram and offsets from the routing record, places its own token's
 // pairs and copies the token's row to them; block 0 also publishes the batch description.
@@ -846,6 +943,23 @@ cudaError_t launch_router_small(const bf16* x, const bf16* Wg, int T, int h, int
     default: return launch_pdl(router_small_kernel<kMaxE>, dim3(T), dim3(256), 0, st, x, Wg, T, h, r, beta, kept, out);
   }
   return cudaGetLastError();
+}
+
+cudaError_t launch_route_single(const bf16* x, const bf16* Wg, int h, int r, float beta,
+                                const KeptIds& kept, const RouteOut& out, int pad, Meta* meta,
+                                int32_t* pair_pos, int32_t* row_token, bf16* xperm, int32_t* s_count,
+                                int32_t* s_nskipped, int32_t* s_ntouched, int E, cudaStream_t st) {
+#define MOE_ROUTE_SINGLE(R)                                                                        \
+  return launch_pdl(route_single_kernel<R>, dim3(1), dim3(256), 0, st, x, Wg, h, r, beta, kept, out, \
+                    pad, meta, pair_pos, row_token, xperm, s_count, s_nskipped, s_ntouched, E)
+  switch (r) {
+    case 2: MOE_ROUTE_SINGLE(2);
+    case 3: case 4: MOE_ROUTE_SINGLE(4);
+    case 5: case 6: MOE_ROUTE_SINGLE(6);
+    case 7: case 8: MOE_ROUTE_SINGLE(8);
+    default: MOE_ROUTE_SINGLE(kMaxE);
+  }
+#undef MOE_ROUTE_SINGLE
 }
 
 cudaError_t launch_permute_gather_small(const bf16* x, const int32_t* idx, const uint8_t* skipped, int T,
