@@ -157,9 +157,12 @@ inline int rows_for(const moe_layer* L, int T, int k = 2) {
   const int pad = decode_mode(T) ? 16 : kTileRows;
   return (int)align_up((size_t)k * T + (size_t)L->r * pad, 16);
 }
-inline int ksplit_for(const moe_layer* L) {
+// k-blocks per work item of the small-batch down projection: with one or two tokens at most four
+// experts are touched, and finer items spread their few weight tiles over more SMs
+inline int down_kb_per_item(int T) { return T <= 2 ? (kDecodeKbPerItem + 1) / 2 : kDecodeKbPerItem; }
+inline int ksplit_for(const moe_layer* L, int T) {
   const int KB = (L->f + 63) / 64;
-  return (KB + kDecodeKbPerItem - 1) / kDecodeKbPerItem;
+  return (KB + down_kb_per_item(T) - 1) / down_kb_per_item(T);
 }
 
 int build_token_maps(GemmMaps& m, const void* base, uint64_t inner, uint64_t rows) {
@@ -173,7 +176,7 @@ int ensure_gemm(moe_layer* L, int T, int k = 2) {
   // capacity in rows: large enough for this T in its mode, at least 256 (TMA boxes)
   int need = (int)align_up((size_t)rows_for(L, T, k), kTileRows) + kTileRows;
   if (need < 256) need = 256;
-  size_t need_O = (size_t)need * L->h * (decode_mode(T) ? ksplit_for(L) : 1);
+  size_t need_O = (size_t)need * L->h * (decode_mode(T) ? ksplit_for(L, T) : 1);
   if (need <= L->ws->cap_rows && need_O * 4 <= L->ws->O.bytes && L->ws->map_h == L->h &&
       L->ws->map_f == L->f)
     return MOE_OK;
@@ -226,7 +229,7 @@ int check_status(moe_layer* L) {
 // The two grouped GEMMs of the experts over a batch described by `meta`.
 int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmMaps& m_gu,
                      const GemmMaps& m_dn, GemmArgs gu, GemmArgs dn, GemmOut dn_kind,
-                     const bf16* gu_A, const bf16* dn_A, int simt_rows) {
+                     const bf16* gu_A, const bf16* dn_A, int simt_rows, int T = 0) {
   gu.meta = meta; dn.meta = meta;
   gu.r = L->r; dn.r = L->r;
   gu.K = L->h; gu.n_w_rows = 2 * L->f;
@@ -239,7 +242,7 @@ int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmM
   } else if (weights_m) {
     CUDA_TRY(launch_gemm_weights_m(true, m_gu, gu, (L->h + 63) / 64, L->stream));
     mark(L);
-    CUDA_TRY(launch_gemm_weights_m(false, m_dn, dn, kDecodeKbPerItem, L->stream));
+    CUDA_TRY(launch_gemm_weights_m(false, m_dn, dn, down_kb_per_item(T), L->stream));
   } else {
     CUDA_TRY(launch_gemm_tokens_m(true, kOutActBf16, m_gu, gu, L->stream));
     mark(L);
@@ -314,7 +317,7 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   if (wm) {
     gu.tail = (float*)L->ws->tail.p; dn.tail = (float*)L->ws->tail.p;
   }
-  const int ksplit = wm ? ksplit_for(L) : 1;
+  const int ksplit = wm ? ksplit_for(L, T) : 1;
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;
   GemmMaps m_gu, m_dn;
@@ -323,7 +326,7 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   memcpy(m_gu.t, L->ws->tok_x, sizeof(m_gu.t));
   memcpy(m_dn.t, L->ws->tok_act, sizeof(m_dn.t));
   rc = run_expert_gemms(L, meta, wm, m_gu, m_dn, gu, dn, kOutF32, (const bf16*)L->ws->xperm.p,
-                        (const bf16*)L->ws->act.p, rows_cap);
+                        (const bf16*)L->ws->act.p, rows_cap, T);
   if (rc) return rc;
   mark(L);
   if (dist)
@@ -531,7 +534,7 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
   if (wm) {
     gu.tail = (float*)W.tail.p; dn.tail = (float*)W.tail.p;
   }
-  const int ksplit = wm ? ksplit_for(L) : 1;
+  const int ksplit = wm ? ksplit_for(L, T) : 1;
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;
   GemmMaps m_gu, m_dn;
@@ -542,7 +545,7 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
   const bool prof_saved = L->prof;
   L->prof = false;
   rc = run_expert_gemms(L, meta, wm, m_gu, m_dn, gu, dn, kOutF32, (const bf16*)W.xperm.p,
-                        (const bf16*)W.act.p, rows_cap);
+                        (const bf16*)W.act.p, rows_cap, T);
   L->prof = prof_saved;
   if (rc) return rc;
   CUDA_TRY(launch_combine_topk((const float*)W.O.p, ksplit, split_stride, (int32_t*)W.k_pos.p,
