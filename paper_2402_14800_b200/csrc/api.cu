@@ -89,6 +89,7 @@ struct moe_layer {
   size_t weight_bytes = 0;
   cudaStream_t stream = 0;
   bool debug_simt = false;
+  int decode_kernel = 0;  // small batches: 0 = by batch size, 1 = weight-major, 2 = token-major (MOE_DECODE_KERNEL=wm|td)
   bool search_dense = false;  // MOE_SEARCH_DENSE=1: evaluate all E experts per token in the search
   CUtensorMap w13_256, w13_128, w2_256, w2_128;
   Workspace own;
@@ -153,6 +154,11 @@ int ensure_route(moe_layer* L, int T) {
 }
 
 inline bool decode_mode(int T) { return T <= kDecodeMaxT; }
+// Small batches run the weight-major GEMM up to kTokensDFromT - 1 tokens and the token-major
+// decode GEMM from there on (measured crossover), unless the handle was told otherwise.
+inline bool decode_weights_m(const moe_layer* L, int T) {
+  return L->decode_kernel == 1 || (L->decode_kernel == 0 && T < kTokensDFromT);
+}
 inline int rows_for(const moe_layer* L, int T, int k = 2) {
   const int pad = decode_mode(T) ? 16 : kTileRows;
   return (int)align_up((size_t)k * T + (size_t)L->r * pad, 16);
@@ -239,10 +245,14 @@ int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmM
     CUDA_TRY(launch_simt_gate_up(gu_A, L->W13, gu, simt_rows, L->stream));
     mark(L);
     CUDA_TRY(launch_simt_down(dn_A, L->W2, dn, simt_rows, dn_kind, L->stream));
-  } else if (weights_m) {
+  } else if (weights_m && decode_weights_m(L, T)) {
     CUDA_TRY(launch_gemm_weights_m(true, m_gu, gu, (L->h + 63) / 64, L->stream));
     mark(L);
     CUDA_TRY(launch_gemm_weights_m(false, m_dn, dn, down_kb_per_item(T), L->stream));
+  } else if (weights_m) {
+    CUDA_TRY(launch_gemm_tokens_d(true, m_gu, gu, (L->h + 63) / 64, L->stream));
+    mark(L);
+    CUDA_TRY(launch_gemm_tokens_d(false, m_dn, dn, down_kb_per_item(T), L->stream));
   } else {
     CUDA_TRY(launch_gemm_tokens_m(true, kOutActBf16, m_gu, gu, L->stream));
     mark(L);
@@ -321,8 +331,8 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;
   GemmMaps m_gu, m_dn;
-  m_gu.w = (wm || gemm_pair_mode()) ? L->w13_128 : L->w13_256;
-  m_dn.w = (wm || gemm_pair_mode()) ? L->w2_128 : L->w2_256;
+  m_gu.w = (wm ? decode_weights_m(L, T) : gemm_pair_mode()) ? L->w13_128 : L->w13_256;
+  m_dn.w = (wm ? decode_weights_m(L, T) : gemm_pair_mode()) ? L->w2_128 : L->w2_256;
   memcpy(m_gu.t, L->ws->tok_x, sizeof(m_gu.t));
   memcpy(m_dn.t, L->ws->tok_act, sizeof(m_dn.t));
   rc = run_expert_gemms(L, meta, wm, m_gu, m_dn, gu, dn, kOutF32, (const bf16*)L->ws->xperm.p,
@@ -401,6 +411,8 @@ moe_layer_t* moe_layer_create(const void* W_gate, const void* W1, const void* W3
   for (int c = L->r; c < kMaxE; ++c) L->kept.id[c] = 0;
   const char* dbg = getenv("MOE_DEBUG_SIMT");
   L->debug_simt = dbg && dbg[0] == '1';
+  const char* dk = getenv("MOE_DECODE_KERNEL");
+  L->decode_kernel = (dk && !strcmp(dk, "wm")) ? 1 : ((dk && !strcmp(dk, "td")) ? 2 : 0);
   const char* nopdl = getenv("MOE_NO_PDL");
   if (nopdl) g_pdl_enabled = nopdl[0] != '1';
   const char* pair = getenv("MOE_GEMM_PAIR");
@@ -538,8 +550,8 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;
   GemmMaps m_gu, m_dn;
-  m_gu.w = (wm || gemm_pair_mode()) ? L->w13_128 : L->w13_256;
-  m_dn.w = (wm || gemm_pair_mode()) ? L->w2_128 : L->w2_256;
+  m_gu.w = (wm ? decode_weights_m(L, T) : gemm_pair_mode()) ? L->w13_128 : L->w13_256;
+  m_dn.w = (wm ? decode_weights_m(L, T) : gemm_pair_mode()) ? L->w2_128 : L->w2_256;
   memcpy(m_gu.t, W.tok_x, sizeof(m_gu.t));
   memcpy(m_dn.t, W.tok_act, sizeof(m_dn.t));
   const bool prof_saved = L->prof;

@@ -17,7 +17,8 @@ constexpr int kTileRows = 128;            // token rows per row tile of the grou
 constexpr int kRouteTokPerBlock = 16;     // tokens routed by one block (one warp per token)
 constexpr int kHistCols = 2 * kMaxE + 1;  // per (expert, slot) pair counts + skipped count
 constexpr int kInterleave = 16;           // W1/W3 rows are interleaved in groups of 16
-constexpr int kDecodeMaxT = 256;          // up to here the weight-stationary GEMM is used
+constexpr int kDecodeMaxT = 256;          // up to here the small-batch path (weights read once) is used
+constexpr int kTokensDFromT = 48;         // small batches from this size on: token-major decode GEMM
 #ifndef MOE_DOWN_KB
 #define MOE_DOWN_KB 112
 #endif
@@ -193,6 +194,8 @@ struct GemmMaps {
 cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps& maps,
                                  const GemmArgs& a, cudaStream_t st);
 // Weight rows are the 128-row MMA operand, tokens the narrow one (small T): weights stream once.
+cudaError_t launch_gemm_tokens_d(bool gate_up, const GemmMaps& maps, const GemmArgs& a, int kb_per_item,
+                                 cudaStream_t st);
 cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
                                   int kb_per_item, cudaStream_t st);
 // Plain CUDA-core kernels of the same contractions, for bring-up and debugging only

@@ -785,13 +785,15 @@ constexpr int kFoldLoads = MOE_FOLD_LOADS;         // tokens x slices one thread
 constexpr int kTailHeaderFloats = (int)(kTailHeaderBytes / 4);  // arrival counters come first
 
 // Warp-collective: all 32 lanes of a converged warp call it and get the same result.
+// tile_w = weight rows of an item (128 weight-major, 256 token-major); a partial tile holds
+// tile_w floats per token; kst_cap bounds the slices by what the fold may load per thread.
 __device__ __forceinline__ SchedW make_sched_w(const Meta& m, const GemmArgs& a, int kb_per_item,
-                                               int grid) {
+                                               int grid, int tile_w = 128, int kst_cap = 0) {
   SchedW s;
   s.KB = (a.K + BK - 1) / BK;
   s.kb_per_item = kb_per_item;
   s.KS = (s.KB + kb_per_item - 1) / kb_per_item;
-  s.Mt = (a.n_w_rows + 127) / 128;
+  s.Mt = (a.n_w_rows + tile_w - 1) / tile_w;
   s.n_base = m.tile_prefix[a.r] * s.Mt * s.KS;
   s.full = (s.n_base / grid) * grid;
   s.rem = s.n_base - s.full;
@@ -800,10 +802,10 @@ __device__ __forceinline__ SchedW make_sched_w(const Meta& m, const GemmArgs& a,
   int maxcnt = 1;
   for (int c = 0; c < a.r; ++c) maxcnt = max(maxcnt, min(m.count[c], WM_BN));
   const int slot_tokens = (maxcnt + 15) & ~15;
-  s.slot_floats = 128 * slot_tokens;
+  s.slot_floats = tile_w * slot_tokens;
   if (a.tail != nullptr && s.rem > 0) {
     const int n_slots = (int)((kTailBufferBytes - kTailHeaderBytes) / ((size_t)s.slot_floats * 4));
-    const int kst_fold = kFoldLoads / slot_tokens;
+    const int kst_fold = kst_cap > 0 ? kst_cap : kFoldLoads / slot_tokens;
     const int want = (int)(threadIdx.x & 31) + 1;  // this lane tries `want` slices per item
     const int kbs = (kb_per_item + want - 1) / want;
     const int kst = (kb_per_item + kbs - 1) / kbs;
@@ -1094,6 +1096,233 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   teardown<WM_NS, 256>(bars, tmem_base, issued, args.status);
 }
 
+// ----------------------------------------------------------------------- gemm_tokens_d
+//
+// Small batches (T <= 256), token-major: every tcgen05.mma costs the same ~140 cycles whatever
+// its M and N, so the weights go where an instruction holds the most of them: the N operand,
+// 256 weight rows x 16 k (8 KB) per instruction against 4 KB when they are the M operand.  The
+// token tile is the M operand: only the rows the expert really has are loaded (boxes of 16 to
+// 128 rows), the rest of its 128-row slot keeps stale data whose accumulator rows are never
+// stored.  Work items, the K-slices of the remainder that run first and their fold are those of
+// the weight-major kernel, with 256-row weight tiles.
+
+constexpr int TD_NS = 4;
+constexpr int TD_A_BYTES = 128 * 128;  // slot of the token tile (16 .. 128 rows loaded)
+constexpr int TD_B_BYTES = 256 * 128;  // 256 weight rows x 64 bf16
+constexpr int TD_STAGE = TD_A_BYTES + TD_B_BYTES;
+constexpr int TD_SMEM = TD_NS * TD_STAGE + 1024;
+constexpr int TD_BN = 256;
+constexpr int kFoldSlicesD = 8;  // the fold of this kernel reads 256 floats per slice and token
+
+// 32 accumulator columns of one token row -> output (SwiGLU + bf16, or fp32), as in
+// store_tile_tokens_m.  col0 = first weight row of the chunk, orow = element offset of the row.
+template <bool GATE_UP>
+__device__ __forceinline__ void store_chunk_d(const float* v, const GemmArgs& args, long long orow, int col0) {
+  if (GATE_UP) {
+    uint32_t o[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      o[i] = pack_bf16(silu_mul(v[2 * i], v[16 + 2 * i]), silu_mul(v[2 * i + 1], v[17 + 2 * i]));
+    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(args.out) + orow + (col0 >> 1));
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+  } else {
+    float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.out) + orow + col0);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+  }
+}
+
+template <bool GATE_UP>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tokens_d_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args, int kb_per_item) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ Bars bars;
+  __shared__ Meta s_meta;
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  setup_barriers<TD_NS>(bars);
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars.tmem_base), 512);
+    tmem_relinquish();
+  }
+  // Rows of the token slots that no load ever writes feed the tensor core all the same: start
+  // them at zero (multiplying zeros costs far less power than multiplying stale data).
+  {
+    uint8_t* gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    for (int s = 0; s < TD_NS; ++s)
+      for (int i = threadIdx.x; i < TD_A_BYTES / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(gen + s * TD_STAGE)[i] = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async();
+  }
+  pdl_wait();
+  for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
+    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *(volatile uint32_t*)&bars.tmem_base;
+  volatile int* abort_flag = &bars.abort_flag;
+
+  const SchedW sched = make_sched_w(s_meta, args, kb_per_item, (int)gridDim.x, TD_BN, kFoldSlicesD);
+  const int n_items = sched.n_total;
+  uint32_t issued = 0;
+
+  if (warp == 0) {
+    uint32_t it = 0;
+    bool ok = true;
+    const uint64_t evict_first = l2_policy_evict_first();
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      ItemW w;
+      decode_item_w(s_meta, args, sched, item, w);
+      if (w.kb0 >= w.kb1) continue;
+      const uint32_t bytes = TD_B_BYTES + (16u << w.bucket) * 128u;
+      for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+        const uint32_t s = it % TD_NS, ph = (it / TD_NS) & 1u;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag));
+        if (!ok) break;
+        if (lane == 0) {
+          const uint32_t full = smem_u32(&bars.full[s]);
+          const uint32_t sa = smem_base + s * TD_STAGE;
+          mbar_expect_tx(full, bytes);
+          tma_load_3d_hint(sa + TD_A_BYTES, &maps.w, kb * BK, w.mt * TD_BN, w.c, full, evict_first);
+          tma_load_2d(sa, &maps.t[w.bucket], kb * BK, w.tok_row, full);
+        }
+        __syncwarp();
+      }
+    }
+    issued = it;
+  } else if (warp == 1) {
+    uint32_t it = 0, tile_it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      ItemW w;
+      decode_item_w(s_meta, args, sched, item, w);
+      if (w.kb0 >= w.kb1) continue;
+      // up to 64 token rows: the M = 64 form (same issue time, half the multiplications)
+      const uint32_t idesc = idesc_bf16(w.cnt <= 64 ? 64 : 128, TD_BN);
+      const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_empty[buf]), bph ^ 1u, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + buf * TD_BN;
+      for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+        const uint32_t s = it % TD_NS, ph = (it / TD_NS) & 1u;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t sa = smem_base + s * TD_STAGE;
+          const uint64_t adesc = smem_desc_k128(sa);
+          const uint64_t bdesc = smem_desc_k128(sa + TD_A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
+          umma_commit(smem_u32(&bars.empty[s]));
+          if (kb == w.kb1 - 1) umma_commit(smem_u32(&bars.tmem_full[buf]));
+        }
+        __syncwarp();
+      }
+      ++tile_it;
+    }
+  } else {
+    // epilogue warp wq reads tensor-memory lanes 32 wq .. 32 wq + 31.  M = 128: lane l of the
+    // tile is token row l.  M = 64: rows 16 q .. 16 q + 15 sit in lanes 32 q .. 32 q + 15.
+    const int wq = warp & 3;
+    uint32_t tile_it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      ItemW w;
+      decode_item_w(s_meta, args, sched, item, w);
+      if (w.kb0 >= w.kb1) continue;
+      const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_full[buf]), bph, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      ++tile_it;
+      const uint32_t taddr = tmem_base + ((uint32_t)(32 * wq) << 16) + buf * TD_BN;
+      const bool m64 = w.cnt <= 64;
+      const int row = m64 ? 16 * wq + lane : 32 * wq + lane;
+      const bool warp_has_rows = (m64 ? 16 * wq : 32 * wq) < w.cnt;  // warp-uniform
+      const bool row_ok = row < w.cnt && (!m64 || lane < 16);
+      const long long orow = (long long)(w.out_row + row) * args.out_ld +
+                             (GATE_UP ? 0ll : (long long)w.ks * args.split_stride);
+      const int nchunk = min(TD_BN, args.n_w_rows - w.mt * TD_BN) / 32;  // 32-column chunks in range
+      if (w.tail_slot < 0) {
+        if (warp_has_rows) {
+#pragma unroll 1
+          for (int j = 0; j < nchunk; ++j) {
+            uint32_t v[32];
+            tmem_ld32(taddr + 32 * j, v);
+            tmem_ld_wait();
+            if (row_ok) store_chunk_d<GATE_UP>(reinterpret_cast<const float*>(v), args, orow, w.mt * TD_BN + 32 * j);
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[buf]));
+        continue;
+      }
+      // K-slice of a tail item: fp32 partial tile [token][256 weight rows]
+      float* slots = args.tail + kTailHeaderFloats;
+      if (warp_has_rows) {
+        float4* outp = reinterpret_cast<float4*>(slots + (size_t)w.tail_slot * sched.slot_floats + row * TD_BN);
+#pragma unroll 1
+        for (int j = 0; j < nchunk; ++j) {
+          uint32_t v[32];
+          tmem_ld32(taddr + 32 * j, v);
+          tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              outp[8 * j + i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                            __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[buf]));
+      if (!warp_has_rows) continue;
+      // the warp that arrives last for these 32 token rows of the item folds them
+      __threadfence();
+      __syncwarp();
+      int* counter = reinterpret_cast<int*>(args.tail) + w.tail_item * 4 + wq;
+      int last = 0;
+      if (lane == 0) last = atomicAdd(counter, 1) == w.nslice - 1;
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (!last) continue;
+      __threadfence();
+      if (row_ok) {
+        const float* src = slots + (size_t)(w.tail_item * sched.KSt) * sched.slot_floats + row * TD_BN;
+#pragma unroll 1
+        for (int j = 0; j < nchunk; ++j) {
+          float v[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = 0.f;
+#pragma unroll 2
+          for (int sub = 0; sub < w.nslice; ++sub) {
+            const float4* p = reinterpret_cast<const float4*>(src + (size_t)sub * sched.slot_floats + 32 * j);
+            float4 q[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) q[i] = __ldcg(p + i);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              v[4 * i] += q[i].x; v[4 * i + 1] += q[i].y; v[4 * i + 2] += q[i].z; v[4 * i + 3] += q[i].w;
+            }
+          }
+          store_chunk_d<GATE_UP>(v, args, orow, w.mt * TD_BN + 32 * j);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) *counter = 0;  // ready for the next launch
+    }
+  }
+  pdl_launch_dependents();
+  teardown<TD_NS, 512>(bars, tmem_base, issued, args.status);
+}
+
 // ------------------------------------------------------------ CUDA-core debug kernels
 
 __device__ __forceinline__ float dot8(const uint4& a, const uint4& b, float acc) {
@@ -1217,6 +1446,8 @@ cudaError_t gemm_set_attributes() {
   SET_ATTR((gemm_tokens_m2_kernel<false, kOutBf16>), T2_SMEM)
   SET_ATTR((gemm_weights_m_kernel<true>), WM_SMEM)
   SET_ATTR((gemm_weights_m_kernel<false>), WM_SMEM)
+  SET_ATTR((gemm_tokens_d_kernel<true>), TD_SMEM)
+  SET_ATTR((gemm_tokens_d_kernel<false>), TD_SMEM)
 #undef SET_ATTR
   int dev = 0;
   e = cudaGetDevice(&dev);
@@ -1264,6 +1495,16 @@ cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps&
   if (out_kind == kOutF32)
     return launch_plain(gemm_tokens_m_kernel<false, kOutF32>, dim3(grid), dim3(kThreads), TM_SMEM, st, maps, a);
   return launch_plain(gemm_tokens_m_kernel<false, kOutBf16>, dim3(grid), dim3(kThreads), TM_SMEM, st, maps, a);
+}
+
+cudaError_t launch_gemm_tokens_d(bool gate_up, const GemmMaps& maps, const GemmArgs& a, int kb_per_item,
+                                 cudaStream_t st) {
+  const int grid = g_num_sms > 0 ? g_num_sms : 148;
+  if (gate_up)
+    return launch_pdl(gemm_tokens_d_kernel<true>, dim3(grid), dim3(kThreads), TD_SMEM, st, maps, a,
+                      kb_per_item);
+  return launch_pdl(gemm_tokens_d_kernel<false>, dim3(grid), dim3(kThreads), TD_SMEM, st, maps, a,
+                    kb_per_item);
 }
 
 cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,

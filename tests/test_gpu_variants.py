@@ -54,6 +54,25 @@ def test_debug_cuda_core_kernels_agree_with_tensor_core_path(weights, T):
     dbg.close()
 
 
+@pytest.mark.parametrize("T", [1, 5, 40, 150, 256])
+def test_both_small_batch_gemms_at_every_size(weights, T):
+    # by default the batch size picks the kernel of a small batch; each one is forced here over
+    # the whole range and compared with the CUDA-core kernels
+    x = synth.make_tokens(T, H, seed=6).to(DEV)
+    dbg = layer_with_env(weights, 0b01111011, MOE_DEBUG_SIMT=1)
+    y0 = dbg.forward(x, 0.3)
+    for kernel in ("wm", "td"):
+        lay = layer_with_env(weights, 0b01111011, MOE_DECODE_KERNEL=kernel)
+        y1 = lay.forward(x, 0.3)
+        y2 = lay.forward(x, 0.3)
+        torch.cuda.synchronize()
+        assert rel_l2(y1, y0) < 5e-3
+        assert torch.equal(y1, y2)
+        assert lay.device_status() == 0
+        lay.close()
+    dbg.close()
+
+
 @pytest.mark.parametrize("r", [6, 4, 7])
 def test_dense_search_equals_pruned_work_search(weights, r):
     x = synth.make_tokens(777, H, seed=4).to(DEV)
