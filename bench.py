@@ -384,7 +384,11 @@ def run_ours(a):
             gu_bytes = touched * 2 * F * H * 2 + pairs * H * 2 + pairs * F * 2
             dn_bytes = touched * H * F * 2 + pairs * F * 2 + 2 * pairs * H * 4
             ach = gu_bytes / (gu_ms * 1e-3) / 1e9
-            roofline = {"bound": "hbm", "kernel": "gemm_weights_m_kernel<gate_up>", "achieved": ach,
+            forced = os.environ.get("MOE_DECODE_KERNEL", "")
+            token_major = forced == "td" or (forced != "wm" and a.tokens >= 48)  # the library's crossover
+            roofline = {"bound": "hbm",
+                        "kernel": "gemm_tokens_d_kernel<gate_up>" if token_major else "gemm_weights_m_kernel<gate_up>",
+                        "achieved": ach,
                         "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"],
                         "traffic": recorded_traffic(workload_name(a)),
                         "peak_source": peaks["source"], "algorithmic_bytes": gu_bytes,
