@@ -1098,13 +1098,15 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
 
 // ----------------------------------------------------------------------- gemm_tokens_d
 //
-// Small batches (T <= 256), token-major: every tcgen05.mma costs the same ~140 cycles whatever
-// its M and N, so the weights go where an instruction holds the most of them: the N operand,
-// 256 weight rows x 16 k (8 KB) per instruction against 4 KB when they are the M operand.  The
-// token tile is the M operand: only the rows the expert really has are loaded (boxes of 16 to
-// 128 rows), the rest of its 128-row slot keeps stale data whose accumulator rows are never
-// stored.  Work items, the K-slices of the remainder that run first and their fold are those of
-// the weight-major kernel, with 256-row weight tiles.
+// Small batches (T <= 256), token-major.  The warp that issues the MMAs spends about 550 cycles
+// per k-block whatever the tile (four instructions of ~57 cycles each when N <= 64, a commit of
+// ~120, the barrier wait and fences), which bounds an SM of the weight-major kernel at 16 KB of
+// weights per k-block.  With the weights as the N operand a k-block carries 256 rows = 32 KB
+// (four instructions of 128 cycles), twice the bytes per trip round the loop.  The token tile is
+// the M operand: only the rows the expert really has are loaded (boxes of 16 to 128 rows), the
+// rest of its 128-row slot is zero and its accumulator rows are never stored.  Work items, the
+// K-slices of the remainder that run first and their fold are those of the weight-major kernel,
+// with 256-row weight tiles.
 
 constexpr int TD_NS = 4;
 constexpr int TD_A_BYTES = 128 * 128;  // slot of the token tile (16 .. 128 rows loaded)
@@ -1200,7 +1202,7 @@ gemm_tokens_d_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args,
       ItemW w;
       decode_item_w(s_meta, args, sched, item, w);
       if (w.kb0 >= w.kb1) continue;
-      // up to 64 token rows: the M = 64 form (same issue time, half the multiplications)
+      // up to 64 token rows: the M = 64 form (half the multiplications, hence less board power)
       const uint32_t idesc = idesc_bf16(w.cnt <= 64 ? 64 : 128, TD_BN);
       const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_empty[buf]), bph ^ 1u, abort_flag));
