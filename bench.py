@@ -385,7 +385,9 @@ def run_ours(a):
             dn_bytes = touched * H * F * 2 + pairs * F * 2 + 2 * pairs * H * 4
             ach = gu_bytes / (gu_ms * 1e-3) / 1e9
             forced = os.environ.get("MOE_DECODE_KERNEL", "")
-            token_major = forced == "td" or (forced != "wm" and a.tokens >= 48)  # the library's crossover
+            r_kept = bin(KEPT[a.kept]).count("1")
+            # the library's crossover: many tokens per expert -> token-major decode kernel
+            token_major = forced == "td" or (forced != "wm" and 2 * a.tokens >= 40 * r_kept)
             roofline = {"bound": "hbm",
                         "kernel": "gemm_tokens_d_kernel<gate_up>" if token_major else "gemm_weights_m_kernel<gate_up>",
                         "achieved": ach,

@@ -154,10 +154,10 @@ int ensure_route(moe_layer* L, int T) {
 }
 
 inline bool decode_mode(int T) { return T <= kDecodeMaxT; }
-// Small batches run the weight-major GEMM up to kTokensDFromT - 1 tokens and the token-major
-// decode GEMM from there on (measured crossover), unless the handle was told otherwise.
+// Small batches run the weight-major GEMM unless the experts hold many tokens each (about
+// 2T/r): from kTokensDPerExpert on, the token-major decode GEMM is faster (measured crossover).
 inline bool decode_weights_m(const moe_layer* L, int T) {
-  return L->decode_kernel == 1 || (L->decode_kernel == 0 && T < kTokensDFromT);
+  return L->decode_kernel == 1 || (L->decode_kernel == 0 && 2 * T < kTokensDPerExpert * L->r);
 }
 inline int rows_for(const moe_layer* L, int T, int k = 2) {
   const int pad = decode_mode(T) ? 16 : kTileRows;
@@ -246,9 +246,9 @@ int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmM
     mark(L);
     CUDA_TRY(launch_simt_down(dn_A, L->W2, dn, simt_rows, dn_kind, L->stream));
   } else if (weights_m && decode_weights_m(L, T)) {
-    CUDA_TRY(launch_gemm_weights_m(true, m_gu, gu, (L->h + 63) / 64, L->stream));
+    CUDA_TRY(launch_gemm_weights_m(true, m_gu, gu, (L->h + 63) / 64, T, L->stream));
     mark(L);
-    CUDA_TRY(launch_gemm_weights_m(false, m_dn, dn, down_kb_per_item(T), L->stream));
+    CUDA_TRY(launch_gemm_weights_m(false, m_dn, dn, down_kb_per_item(T), T, L->stream));
   } else if (weights_m) {
     CUDA_TRY(launch_gemm_tokens_d(true, m_gu, gu, (L->h + 63) / 64, L->stream));
     mark(L);

@@ -18,7 +18,7 @@ constexpr int kRouteTokPerBlock = 16;     // tokens routed by one block (one war
 constexpr int kHistCols = 2 * kMaxE + 1;  // per (expert, slot) pair counts + skipped count
 constexpr int kInterleave = 16;           // W1/W3 rows are interleaved in groups of 16
 constexpr int kDecodeMaxT = 256;          // up to here the small-batch path (weights read once) is used
-constexpr int kTokensDFromT = 48;         // small batches from this size on: token-major decode GEMM
+constexpr int kTokensDPerExpert = 40;      // small batches with this many tokens per expert or more: token-major decode GEMM
 #ifndef MOE_DOWN_KB
 #define MOE_DOWN_KB 112
 #endif
@@ -197,7 +197,7 @@ cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps&
 cudaError_t launch_gemm_tokens_d(bool gate_up, const GemmMaps& maps, const GemmArgs& a, int kb_per_item,
                                  cudaStream_t st);
 cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
-                                  int kb_per_item, cudaStream_t st);
+                                  int kb_per_item, int max_tokens_per_tile, cudaStream_t st);
 // Plain CUDA-core kernels of the same contractions, for bring-up and debugging only
 // (MOE_DEBUG_SIMT=1); never selected otherwise.
 cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,

@@ -739,14 +739,18 @@ gemm_tokens_m2_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
 
 // ----------------------------------------------------------------------- gemm_weights_m
 
-#ifndef MOE_WM_NS
-#define MOE_WM_NS 6
-#endif
-constexpr int WM_NS = MOE_WM_NS;
+// A pipeline stage holds two k-blocks (one barrier wait and one commit per 32 KB of weights: the
+// loop of the MMA-issuing warp, not memory, bounds this kernel):
+//   [weights kb][weights kb+1][tokens kb][tokens kb+1], token slots of TOK rows.
+// TOK = 64 (batches of at most 64 tokens): 4 stages of 48 KB; TOK = 128: 3 stages of 64 KB.
+// (Smaller slots with more stages were measured: 5 x 40 KB equal, 6 x 36 KB 4-5 % slower.)
 constexpr int WM_A_BYTES = 128 * 128;  // 128 weight rows x 64 bf16
-constexpr int WM_B_BYTES = 128 * 128;  // up to 128 token rows x 64 bf16
-constexpr int WM_STAGE = WM_A_BYTES + WM_B_BYTES;
-constexpr int WM_SMEM = WM_NS * WM_STAGE + 1024;
+template <int TOK> struct WmCfg {
+  static constexpr int kTokBytes = TOK * 128;
+  static constexpr int kStage = 2 * (WM_A_BYTES + kTokBytes);
+  static constexpr int kNS = TOK <= 64 ? 4 : 3;
+  static constexpr int kSmem = kNS * kStage + 1024;
+};
 constexpr int WM_BN = 128;
 
 struct ItemW {
@@ -903,7 +907,7 @@ __device__ __forceinline__ void fold_slices(const GemmArgs& args, const ItemW& w
   }
 }
 
-template <bool GATE_UP>
+template <bool GATE_UP, int TOK>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args, int kb_per_item) {
   extern __shared__ uint8_t smem_raw[];
@@ -912,6 +916,10 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+  using Cfg = WmCfg<TOK>;
+  constexpr int WM_NS = Cfg::kNS;
+  constexpr int WM_STAGE = Cfg::kStage;
+  constexpr int WM_TOK_BYTES = Cfg::kTokBytes;
   setup_barriers<WM_NS>(bars);
   if (warp == 1) {
     tmem_alloc(smem_u32(&bars.tmem_base), 256);
@@ -941,23 +949,26 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
       ItemW w;
       decode_item_w(s_meta, args, sched, item, w);
       if (w.kb0 >= w.kb1) continue;
-      const uint32_t bytes = WM_A_BYTES + (16u << w.bucket) * 128u;
-      for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+      const uint32_t bytes = WM_A_BYTES + (16u << w.bucket) * 128u;  // of one k-block
+      for (int kb = w.kb0; kb < w.kb1; kb += 2, ++it) {
         const uint32_t s = it % WM_NS, ph = (it / WM_NS) & 1u;
+        const int nk = min(2, w.kb1 - kb);
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag));
         if (!ok) break;
         if (lane == 0) {
           const uint32_t full = smem_u32(&bars.full[s]);
           const uint32_t sa = smem_base + s * WM_STAGE;
-          mbar_expect_tx(full, bytes);
+          mbar_expect_tx(full, bytes * nk);
+          for (int j = 0; j < nk; ++j) {
 #ifndef MOE_WM_NO_EVICT_FIRST
-          // every weight byte is read exactly once: do not let it push the token rows, the
-          // activations and the partial sums out of L2
-          tma_load_3d_hint(sa, &maps.w, kb * BK, w.mt * 128, w.c, full, evict_first);
+            // every weight byte is read exactly once: do not let it push the token rows, the
+            // activations and the partial sums out of L2
+            tma_load_3d_hint(sa + j * WM_A_BYTES, &maps.w, (kb + j) * BK, w.mt * 128, w.c, full, evict_first);
 #else
-          tma_load_3d(sa, &maps.w, kb * BK, w.mt * 128, w.c, full);
+            tma_load_3d(sa + j * WM_A_BYTES, &maps.w, (kb + j) * BK, w.mt * 128, w.c, full);
 #endif
-          tma_load_2d(sa + WM_A_BYTES, &maps.t[w.bucket], kb * BK, w.tok_row, full);
+            tma_load_2d(sa + 2 * WM_A_BYTES + j * WM_TOK_BYTES, &maps.t[w.bucket], (kb + j) * BK, w.tok_row, full);
+          }
         }
         __syncwarp();
       }
@@ -976,20 +987,23 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
       if (!ok) break;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + buf * WM_BN;
-      for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+      for (int kb = w.kb0; kb < w.kb1; kb += 2, ++it) {
         const uint32_t s = it % WM_NS, ph = (it / WM_NS) & 1u;
+        const int nk = min(2, w.kb1 - kb);
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag));
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
           const uint32_t sa = smem_base + s * WM_STAGE;
-          const uint64_t adesc = smem_desc_k128(sa);
-          const uint64_t bdesc = smem_desc_k128(sa + WM_A_BYTES);
+          for (int j = 0; j < nk; ++j) {
+            const uint64_t adesc = smem_desc_k128(sa + j * WM_A_BYTES);
+            const uint64_t bdesc = smem_desc_k128(sa + 2 * WM_A_BYTES + j * WM_TOK_BYTES);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)
-            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < BK / UMMA_K; ++k)
+              umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb + j > w.kb0 || k > 0) ? 1u : 0u);
+          }
           umma_commit(smem_u32(&bars.empty[s]));
-          if (kb == w.kb1 - 1) umma_commit(smem_u32(&bars.tmem_full[buf]));
+          if (kb + nk >= w.kb1) umma_commit(smem_u32(&bars.tmem_full[buf]));
         }
         __syncwarp();
       }
@@ -1446,8 +1460,10 @@ cudaError_t gemm_set_attributes() {
   SET_ATTR((gemm_tokens_m2_kernel<true, kOutActBf16>), T2_SMEM)
   SET_ATTR((gemm_tokens_m2_kernel<false, kOutF32>), T2_SMEM)
   SET_ATTR((gemm_tokens_m2_kernel<false, kOutBf16>), T2_SMEM)
-  SET_ATTR((gemm_weights_m_kernel<true>), WM_SMEM)
-  SET_ATTR((gemm_weights_m_kernel<false>), WM_SMEM)
+  SET_ATTR((gemm_weights_m_kernel<true, 64>), WmCfg<64>::kSmem)
+  SET_ATTR((gemm_weights_m_kernel<false, 64>), WmCfg<64>::kSmem)
+  SET_ATTR((gemm_weights_m_kernel<true, 128>), WmCfg<128>::kSmem)
+  SET_ATTR((gemm_weights_m_kernel<false, 128>), WmCfg<128>::kSmem)
   SET_ATTR((gemm_tokens_d_kernel<true>), TD_SMEM)
   SET_ATTR((gemm_tokens_d_kernel<false>), TD_SMEM)
 #undef SET_ATTR
@@ -1509,14 +1525,22 @@ cudaError_t launch_gemm_tokens_d(bool gate_up, const GemmMaps& maps, const GemmA
                     kb_per_item);
 }
 
-cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
-                                  int kb_per_item, cudaStream_t st) {
-  const int grid = g_num_sms > 0 ? g_num_sms : 148;
+template <int TOK>
+static cudaError_t launch_wm(bool gate_up, const GemmMaps& maps, const GemmArgs& a, int kb_per_item, int grid,
+                             cudaStream_t st) {
   if (gate_up)
-    return launch_pdl(gemm_weights_m_kernel<true>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
-                      kb_per_item);
-  return launch_pdl(gemm_weights_m_kernel<false>, dim3(grid), dim3(kThreads), WM_SMEM, st, maps, a,
-                    kb_per_item);
+    return launch_pdl(gemm_weights_m_kernel<true, TOK>, dim3(grid), dim3(kThreads), WmCfg<TOK>::kSmem, st, maps,
+                      a, kb_per_item);
+  return launch_pdl(gemm_weights_m_kernel<false, TOK>, dim3(grid), dim3(kThreads), WmCfg<TOK>::kSmem, st, maps,
+                    a, kb_per_item);
+}
+
+cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
+                                  int kb_per_item, int max_tokens_per_tile, cudaStream_t st) {
+  const int grid = g_num_sms > 0 ? g_num_sms : 148;
+  // no expert group can exceed the batch: small batches take the layout with 64-row token slots
+  if (max_tokens_per_tile <= 64) return launch_wm<64>(gate_up, maps, a, kb_per_item, grid, st);
+  return launch_wm<128>(gate_up, maps, a, kb_per_item, grid, st);
 }
 
 cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,
