@@ -54,12 +54,21 @@ def kernel_source_sha256(kernel: str):
     return hashlib.sha256(src[i:j].encode()).hexdigest()
 
 
-def recorded_traffic(workload: str):
+def single_token_gemv() -> bool:
+    """Whether the library runs a single token through its matrix-vector kernels (its default)
+    rather than the grouped GEMMs (forced by either switch)."""
+    return (os.environ.get("MOE_SINGLE_KERNEL", "") != "gemm"
+            and os.environ.get("MOE_DECODE_KERNEL", "") not in ("wm", "td"))
+
+
+def recorded_traffic(workload: str, kernel: str):
     """DRAM bytes per launch of the dominant kernel from the committed ncu capture of this
-    workload, or None when there is none or that kernel's source changed since."""
+    workload, or None when there is none, it is of another kernel than the one that ran, or
+    that kernel's source changed since."""
     try:
         rec = json.load(open(os.path.join(ROOT, "profiles", "traffic.json"))).get(workload)
-        if rec and kernel_source_sha256(rec["kernel_function"]) == rec["kernel_source_sha256"]:
+        if (rec and rec["kernel"] == kernel
+                and kernel_source_sha256(rec["kernel_function"]) == rec["kernel_source_sha256"]):
             return rec["dram_bytes"]
     except Exception:
         pass
@@ -296,10 +305,12 @@ def run_ours(a):
     else:
         def step():
             layer.forward(x, beta, y=y)
-        # T = 1: routing (one launch), gate/up GEMM, down GEMM, combine;
+        # T = 1: routing (one launch), gate/up matrix-vector kernel, down kernel with the
+        #   weighted sum (with the GEMM path forced: gate/up GEMM, down GEMM, combine);
         # T <= 256: router, permute+gather, gate/up GEMM, down GEMM, combine;
         # larger T: router, scan, scatter, gather, gate/up GEMM, down GEMM, combine
-        launches_per_step = 4 if a.tokens == 1 else (5 if a.tokens <= 256 else 7)
+        single_gemv = a.tokens == 1 and single_token_gemv()
+        launches_per_step = (3 if single_gemv else 4) if a.tokens == 1 else (5 if a.tokens <= 256 else 7)
 
     # routing facts for the algorithmic byte / flop counts (one untimed call)
     pairs = touched = 0
@@ -388,11 +399,12 @@ def run_ours(a):
             r_kept = bin(KEPT[a.kept]).count("1")
             # the library's crossover: many tokens per expert -> token-major decode kernel
             token_major = forced == "td" or (forced != "wm" and 2 * a.tokens >= 40 * r_kept)
-            roofline = {"bound": "hbm",
-                        "kernel": "gemm_tokens_d_kernel<gate_up>" if token_major else "gemm_weights_m_kernel<gate_up>",
-                        "achieved": ach,
+            kernel = "gemm_tokens_d_kernel<gate_up>" if token_major else "gemm_weights_m_kernel<gate_up>"
+            if single_gemv:  # one token: matrix-vector kernels on the CUDA cores
+                kernel = "gemv_gate_up_kernel"
+            roofline = {"bound": "hbm", "kernel": kernel, "achieved": ach,
                         "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"],
-                        "traffic": recorded_traffic(workload_name(a)),
+                        "traffic": recorded_traffic(workload_name(a), kernel),
                         "peak_source": peaks["source"], "algorithmic_bytes": gu_bytes,
                         "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
                         "down_kernel": {"achieved": dn_bytes / (dn_ms * 1e-3) / 1e9,
@@ -404,7 +416,7 @@ def run_ours(a):
             ach = gu_flop / (gu_ms * 1e-3) / 1e12
             roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel<gate_up>", "achieved": ach,
                         "peak": peaks["tf_sust"], "unit": "TFLOP/s", "frac": ach / peaks["tf_sust"],
-                        "traffic": recorded_traffic(workload_name(a)),
+                        "traffic": recorded_traffic(workload_name(a), "gemm_tokens_m_kernel<gate_up>"),
                         "peak_source": peaks["source"] + " (sustained bf16)",
                         "frac_of_burst": ach / peaks["tf_burst"],
                         "frac_of_nominal_dense_bf16": ach / NOMINAL_BF16_TFLOPS,
@@ -639,7 +651,7 @@ def run_stack(a):
                     "frac_of_nominal_dense_bf16": ach / NOMINAL_BF16_TFLOPS,
                     "peak_source": peaks["source"] + " (sustained bf16)"}
     if rank == 0:
-        per_layer = (4 if T == 1 else (5 if T <= 256 else 7)) + 1   # the layer's kernels + its RMSNorm
+        per_layer = ((3 if single_token_gemv() else 4) if T == 1 else (5 if T <= 256 else 7)) + 1   # the layer's kernels + its RMSNorm
         line = {
             "metric": "MoE-stack tokens/s on 1 B200 (32 layers, RMSNorm + residual, attention omitted)",
             "value": value, "unit": "tokens/s", "n_gpus": world, "steps": a.steps,

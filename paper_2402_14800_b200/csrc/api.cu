@@ -90,6 +90,7 @@ struct moe_layer {
   cudaStream_t stream = 0;
   bool debug_simt = false;
   int decode_kernel = 0;  // small batches: 0 = by batch size, 1 = weight-major, 2 = token-major (MOE_DECODE_KERNEL=wm|td)
+  bool single_gemv = true;    // T = 1 runs the matrix-vector kernels (MOE_SINGLE_KERNEL=gemm: the GEMM path)
   bool search_dense = false;  // MOE_SEARCH_DENSE=1: evaluate all E experts per token in the search
   CUtensorMap w13_256, w13_128, w2_256, w2_128;
   Workspace own;
@@ -318,6 +319,18 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
                            (bf16*)L->ws->xperm.p, st));
   mark(L);
 
+  if (T == 1 && L->single_gemv && !L->debug_simt && !dist) {
+    // one token: matrix-vector kernels; the second one also forms the weighted sum and writes y
+    CUDA_TRY(launch_gemv_gate_up((const bf16*)x, L->W13, meta, L->r, L->h, L->f, (bf16*)L->ws->act.p, st));
+    mark(L);
+    CUDA_TRY(launch_gemv_down_combine((const bf16*)L->ws->act.p, L->W2, meta, (int32_t*)L->ws->pair_pos.p,
+                                      (float*)L->ws->wn.p, (const bf16*)residual, L->r, L->h, L->f,
+                                      (bf16*)y, st));
+    mark(L);
+    mark(L);
+    return MOE_OK;
+  }
+
   GemmArgs gu, dn;
   memset(&gu, 0, sizeof(gu));
   memset(&dn, 0, sizeof(dn));
@@ -400,6 +413,7 @@ moe_layer_t* moe_layer_create(const void* W_gate, const void* W1, const void* W3
   if (major != 10) { fail(MOE_ERR_ARCH, "device has compute capability %d.x, sm_100 is required", major); return nullptr; }
   if (gemm_init_driver_api()) { fail(MOE_ERR_CUDA, "cuTensorMapEncodeTiled is not available"); return nullptr; }
   cudaError_t e = gemm_set_attributes();
+  if (e == cudaSuccess) e = gemv_single_setup();
   if (e != cudaSuccess) { fail(MOE_ERR_CUDA, "kernel attributes: %s", cudaGetErrorString(e)); return nullptr; }
 
   moe_layer* L = new (std::nothrow) moe_layer();
@@ -413,6 +427,8 @@ moe_layer_t* moe_layer_create(const void* W_gate, const void* W1, const void* W3
   L->debug_simt = dbg && dbg[0] == '1';
   const char* dk = getenv("MOE_DECODE_KERNEL");
   L->decode_kernel = (dk && !strcmp(dk, "wm")) ? 1 : ((dk && !strcmp(dk, "td")) ? 2 : 0);
+  const char* sk = getenv("MOE_SINGLE_KERNEL");
+  L->single_gemv = !(sk && !strcmp(sk, "gemm")) && L->decode_kernel == 0 && gemv_single_fits(h, f);
   const char* nopdl = getenv("MOE_NO_PDL");
   if (nopdl) g_pdl_enabled = nopdl[0] != '1';
   const char* pair = getenv("MOE_GEMM_PAIR");

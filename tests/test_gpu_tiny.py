@@ -97,6 +97,22 @@ def test_forward_residual_and_beta_above_one(setup):
     run_case(host, dev, 600, FULL, 0.3, residual=True)
 
 
+@pytest.mark.parametrize("kept", [FULL, 0b01100110, 0b00000110])
+@pytest.mark.parametrize("beta", [0.0, 0.45, 1.5])
+def test_forward_single_token(setup, kept, beta):
+    # T = 1 runs the matrix-vector kernels: one or two experts, with and without the residual,
+    # several tokens in turn so that different experts and both skip outcomes occur
+    host, dev = setup
+    skipped = []
+    for seed in range(6):
+        r = run_case(host, dev, 1, kept, beta, x_seed=40 + seed, residual=bool(seed % 2))
+        skipped.append(bool(r["ora"]["skipped"][0]))
+    if beta == 0.0:
+        assert not any(skipped)
+    if beta > 1.0:
+        assert all(skipped)
+
+
 def test_forward_is_deterministic_and_reuses_scratch(setup):
     host, dev = setup
     layer = make_layer(dev)
@@ -229,6 +245,8 @@ def test_rmsnorm_and_stack(setup):
     (64, 64, 16, 0xFFFF, 513),      # smallest shapes, 16 experts
     (256, 192, 16, 0xF0F3, 200),    # 10 of 16 experts kept (generic router path)
     (128, 448, 2, 0b11, 129),       # every token uses both experts
+    (192, 320, 4, 0b1011, 1),       # single token: matrix-vector kernels, ragged row lengths
+    (64, 64, 16, 0xFFFF, 1),
 ])
 def test_forward_other_shapes(h, f, E, kept, T):
     build.build()

@@ -73,6 +73,25 @@ def test_both_small_batch_gemms_at_every_size(weights, T):
     dbg.close()
 
 
+@pytest.mark.parametrize("beta", [0.0, 0.6])
+def test_single_token_kernels_agree_with_gemm_path(weights, beta):
+    # T = 1 runs matrix-vector kernels by default; MOE_SINGLE_KERNEL=gemm keeps the grouped GEMMs
+    gemv = binding.MoeLayer(*weights, 0b11110110)
+    gemm = layer_with_env(weights, 0b11110110, MOE_SINGLE_KERNEL="gemm")
+    for seed in range(8):
+        x = synth.make_tokens(1, H, seed=50 + seed).to(DEV)
+        res = synth.make_tokens(1, H, seed=90 + seed).to(DEV) if seed % 2 else None
+        y0 = gemm.forward(x, beta, residual=res)
+        y1 = gemv.forward(x, beta, residual=res)
+        y2 = gemv.forward(x, beta, residual=res)
+        torch.cuda.synchronize()
+        assert rel_l2(y1, y0) < 5e-3  # different summation orders, same rounding points
+        assert torch.equal(y1, y2)
+    assert gemv.device_status() == 0 and gemm.device_status() == 0
+    gemv.close()
+    gemm.close()
+
+
 @pytest.mark.parametrize("r", [6, 4, 7])
 def test_dense_search_equals_pruned_work_search(weights, r):
     x = synth.make_tokens(777, H, seed=4).to(DEV)
