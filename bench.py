@@ -305,12 +305,12 @@ def run_ours(a):
     else:
         def step():
             layer.forward(x, beta, y=y)
-        # T = 1: routing (one launch), gate/up matrix-vector kernel, down kernel with the
-        #   weighted sum (with the GEMM path forced: gate/up GEMM, down GEMM, combine);
+        # T = 1: routing + gate/up matrix-vector kernel, down kernel with the weighted sum
+        #   (with the GEMM path forced: routing, gate/up GEMM, down GEMM, combine);
         # T <= 256: router, permute+gather, gate/up GEMM, down GEMM, combine;
         # larger T: router, scan, scatter, gather, gate/up GEMM, down GEMM, combine
         single_gemv = a.tokens == 1 and single_token_gemv()
-        launches_per_step = (3 if single_gemv else 4) if a.tokens == 1 else (5 if a.tokens <= 256 else 7)
+        launches_per_step = (2 if single_gemv else 4) if a.tokens == 1 else (5 if a.tokens <= 256 else 7)
 
     # routing facts for the algorithmic byte / flop counts (one untimed call)
     pairs = touched = 0
@@ -401,7 +401,7 @@ def run_ours(a):
             token_major = forced == "td" or (forced != "wm" and 2 * a.tokens >= 40 * r_kept)
             kernel = "gemm_tokens_d_kernel<gate_up>" if token_major else "gemm_weights_m_kernel<gate_up>"
             if single_gemv:  # one token: matrix-vector kernels on the CUDA cores
-                kernel = "gemv_gate_up_kernel"
+                kernel = "gemv_route_gate_up_kernel"
             roofline = {"bound": "hbm", "kernel": kernel, "achieved": ach,
                         "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"],
                         "traffic": recorded_traffic(workload_name(a), kernel),
@@ -651,7 +651,7 @@ def run_stack(a):
                     "frac_of_nominal_dense_bf16": ach / NOMINAL_BF16_TFLOPS,
                     "peak_source": peaks["source"] + " (sustained bf16)"}
     if rank == 0:
-        per_layer = ((3 if single_token_gemv() else 4) if T == 1 else (5 if T <= 256 else 7)) + 1   # the layer's kernels + its RMSNorm
+        per_layer = ((2 if single_token_gemv() else 4) if T == 1 else (5 if T <= 256 else 7)) + 1   # the layer's kernels + its RMSNorm
         line = {
             "metric": "MoE-stack tokens/s on 1 B200 (32 layers, RMSNorm + residual, attention omitted)",
             "value": value, "unit": "tokens/s", "n_gpus": world, "steps": a.steps,

@@ -297,6 +297,21 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   Meta* meta = (Meta*)L->ws->meta.p;
   if (L->prof && (L->prof_used % (MOE_PROFILE_STAGES + 1)) != 0) L->prof_used = 0;
   mark(L);
+  const bool single_gemv = T == 1 && L->single_gemv && !L->debug_simt && !dist;
+  if (single_gemv) {
+    mark(L);  // (no routing stage of its own)
+    // one token: routing inside the gate/up matrix-vector kernel; the second kernel also forms
+    // the weighted sum and writes y
+    CUDA_TRY(launch_gemv_route_gate_up((const bf16*)x, L->Wg, L->W13, L->r, L->h, L->f, beta, L->kept, ro,
+                                       meta, (int32_t*)L->ws->pair_pos.p, (int32_t*)L->ws->row_token.p,
+                                       s_count, s_nsk, s_nt, L->E, (bf16*)L->ws->act.p, st));
+    mark(L);
+    CUDA_TRY(launch_gemv_down_combine((const bf16*)L->ws->act.p, L->W2, ro.idx, ro.skipped, ro.wn,
+                                      (const bf16*)residual, L->h, L->f, (bf16*)y, st));
+    mark(L);
+    mark(L);
+    return MOE_OK;
+  }
   if (T == 1) {
     CUDA_TRY(launch_route_single((const bf16*)x, L->Wg, L->h, L->r, beta, L->kept, ro, 16, meta,
                                  (int32_t*)L->ws->pair_pos.p, (int32_t*)L->ws->row_token.p,
@@ -318,18 +333,6 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
     CUDA_TRY(launch_gather((const bf16*)x, (int32_t*)L->ws->row_token.p, meta, L->h, rows_cap,
                            (bf16*)L->ws->xperm.p, st));
   mark(L);
-
-  if (T == 1 && L->single_gemv && !L->debug_simt && !dist) {
-    // one token: matrix-vector kernels; the second one also forms the weighted sum and writes y
-    CUDA_TRY(launch_gemv_gate_up((const bf16*)x, L->W13, meta, L->r, L->h, L->f, (bf16*)L->ws->act.p, st));
-    mark(L);
-    CUDA_TRY(launch_gemv_down_combine((const bf16*)L->ws->act.p, L->W2, meta, (int32_t*)L->ws->pair_pos.p,
-                                      (float*)L->ws->wn.p, (const bf16*)residual, L->r, L->h, L->f,
-                                      (bf16*)y, st));
-    mark(L);
-    mark(L);
-    return MOE_OK;
-  }
 
   GemmArgs gu, dn;
   memset(&gu, 0, sizeof(gu));

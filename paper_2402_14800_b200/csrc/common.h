@@ -198,15 +198,18 @@ cudaError_t launch_gemm_tokens_d(bool gate_up, const GemmMaps& maps, const GemmA
                                  cudaStream_t st);
 cudaError_t launch_gemm_weights_m(bool gate_up, const GemmMaps& maps, const GemmArgs& a,
                                   int kb_per_item, int max_tokens_per_tile, cudaStream_t st);
-// Single-token forward on the CUDA cores (matrix-vector kernels, T = 1 only); the second
-// kernel also forms the weighted sum of Eq. 2 and writes y.
+// Single-token forward on the CUDA cores (T = 1 only): routing + gate/up matrix-vector kernel,
+// then the down projection with the weighted sum of Eq. 2, which writes y.
 cudaError_t gemv_single_setup();
 bool gemv_single_fits(int h, int f);
-cudaError_t launch_gemv_gate_up(const bf16* x, const bf16* W13, const Meta* meta, int r, int h, int f,
-                                bf16* act, cudaStream_t st);
-cudaError_t launch_gemv_down_combine(const bf16* act, const bf16* W2, const Meta* meta,
-                                     const int32_t* pair_pos, const float* wn, const bf16* residual,
-                                     int r, int h, int f, bf16* y, cudaStream_t st);
+cudaError_t launch_gemv_route_gate_up(const bf16* x, const bf16* Wg, const bf16* W13, int r, int h, int f,
+                                      float beta, const KeptIds& kept, const RouteOut& ro, Meta* meta,
+                                      int32_t* pair_pos, int32_t* row_token, int32_t* s_count,
+                                      int32_t* s_nskipped, int32_t* s_ntouched, int E, bf16* act,
+                                      cudaStream_t st);
+cudaError_t launch_gemv_down_combine(const bf16* act, const bf16* W2, const int32_t* idx,
+                                     const uint8_t* skipped, const float* wn, const bf16* residual,
+                                     int h, int f, bf16* y, cudaStream_t st);
 // Plain CUDA-core kernels of the same contractions, for bring-up and debugging only
 // (MOE_DEBUG_SIMT=1); never selected otherwise.
 cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& a, int cap_rows,

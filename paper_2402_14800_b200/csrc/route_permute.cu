@@ -7,67 +7,11 @@
 //   gather          copies the routed rows of x into expert-contiguous order.
 //   combine         Eq. 2: y = bf16(residual + w~_e0 o_e0 + w~_e1 o_e1), slot 0 first.
 #include "common.h"
+#include "route_device.cuh"
 
 namespace moe {
 
 namespace {
-
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-
-__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
-  f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x);
-  f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
-  f[4] = bf16_lo(v.z); f[5] = bf16_hi(v.z);
-  f[6] = bf16_lo(v.w); f[7] = bf16_hi(v.w);
-}
-
-__device__ __forceinline__ uint32_t pack2(float a, float b) {
-  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
-  return *reinterpret_cast<uint32_t*>(&p);
-}
-
-// ------------------------------------------------------------------------------- router
-
-// Routing decision of one token from its r logits (one thread); writes the per-token record.
-template <int R>
-__device__ __forceinline__ void route_decide(const float (&acc)[R], int r, float beta, int t,
-                                             const KeptIds& kept, const RouteOut& o, int& e0,
-                                             int& e1, bool& skip) {
-  // top-2 on the logits (softmax is increasing), ties to the lower index
-  e0 = 0;
-  float l0 = acc[0];
-#pragma unroll
-  for (int c = 1; c < R; ++c)
-    if (c < r && acc[c] > l0) { l0 = acc[c]; e0 = c; }
-  e1 = -1;
-  float l1 = 0.f;
-#pragma unroll
-  for (int c = 0; c < R; ++c)
-    if (c < r && c != e0 && (e1 < 0 || acc[c] > l1)) { l1 = acc[c]; e1 = c; }
-  // softmax numerators relative to the maximum: p_e0 = 1, p_e1 = exp(l1 - l0); the
-  // denominator cancels in the ratio, the skip test and the normalised weights
-  const float p1 = expf(l1 - l0);
-  skip = p1 < beta * 1.0f;
-  float w0, w1;
-  if (skip) { w0 = 1.f; w1 = 0.f; }
-  else { const float d = 1.0f + p1; w0 = 1.0f / d; w1 = p1 / d; }
-  o.idx[2 * t] = e0; o.idx[2 * t + 1] = e1;
-  o.wn[2 * t] = w0; o.wn[2 * t + 1] = w1;
-  o.ratio[t] = p1;
-  o.skipped[t] = skip ? 1 : 0;
-  if (o.s_idx) {
-    o.s_idx[2 * t] = kept.id[e0]; o.s_idx[2 * t + 1] = kept.id[e1];
-    o.s_wn[2 * t] = w0; o.s_wn[2 * t + 1] = w1;
-    o.s_ratio[t] = p1;
-    o.s_skipped[t] = skip ? 1 : 0;
-  }
-  if (o.logits) {
-#pragma unroll
-    for (int c = 0; c < R; ++c)
-      if (c < r) o.logits[(size_t)t * r + c] = acc[c];
-  }
-}
 
 // Small batches: one block per token, all loads of a thread independent of each other, so the
 // kernel costs a couple of memory round trips instead of a serial walk over the row.
@@ -172,39 +116,8 @@ route_single_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
     bool skip;
     route_decide<R>(l, r, beta, 0, kept, o, e0, e1, skip);
     if (skip) e1 = -1;
-    // the batch description: one row for e0, one for e1 unless it is skipped
-    int off = 0, tiles = 0;
-    meta->off[0] = 0;
-    meta->tile_prefix[0] = 0;
-    for (int c = 0; c < kMaxE; ++c) {
-      const int n0 = (c == e0), n1 = (c == e1);
-      const int n = n0 + n1;
-      if (c == e0) s_p[0] = off;
-      if (c == e1) s_p[1] = off;
-      off += (n + pad - 1) / pad * pad;
-      tiles += (n + kTileRows - 1) / kTileRows;
-      meta->count[c] = n;
-      meta->count_slot[c][0] = n0;
-      meta->count_slot[c][1] = n1;
-      meta->off[c + 1] = off;
-      meta->tile_prefix[c + 1] = tiles;
-    }
-    if (e1 < 0) s_p[1] = -1;
-    meta->rows_total = off;
-    meta->n_skipped = skip ? 1 : 0;
-    meta->n_touched = skip ? 1 : 2;
-    meta->reserved = 0;
-    pair_pos[0] = s_p[0];
-    pair_pos[1] = s_p[1];
-    row_token[s_p[0]] = 0;
-    if (e1 >= 0) row_token[s_p[1]] = 0;
-    if (s_count) {
-      for (int e = 0; e < E; ++e) { s_count[2 * e] = 0; s_count[2 * e + 1] = 0; }
-      s_count[2 * kept.id[e0]] = 1;
-      if (e1 >= 0) s_count[2 * kept.id[e1] + 1] = 1;
-      *s_nskipped = skip ? 1 : 0;
-      *s_ntouched = skip ? 1 : 2;
-    }
+    publish_single(e0, e1, pad, kept, meta, pair_pos, row_token, s_count, s_nskipped, s_ntouched, E,
+                   s_p[0], s_p[1]);
   }
   __syncthreads();
   const int p0 = s_p[0], p1 = s_p[1];
