@@ -125,7 +125,7 @@ def test_cta_pair_gemm_agrees_with_single_cta_gemm(weights):
     assert b0 == b1
 
 
-@pytest.mark.parametrize("T", [16, 600])
+@pytest.mark.parametrize("T", [1, 16, 600])
 def test_forward_replays_from_a_cuda_graph(weights, T):
     layer = binding.MoeLayer(*weights)
     x = synth.make_tokens(T, H, seed=6).to(DEV)
