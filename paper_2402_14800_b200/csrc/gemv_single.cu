@@ -112,9 +112,8 @@ gemv_route_gate_up_kernel(const bf16* __restrict__ x, const bf16* __restrict__ W
   }
   const int nwarps = gridDim.x * (kGuThreads / 32);
   const int total = (skip ? 1 : 2) * f;
-  // consecutive tasks go to different blocks, so the few tasks of the last, partial round are
-  // spread over the SMs instead of piling up on the first blocks
-  for (int task = warp * gridDim.x + blockIdx.x; task < total; task += nwarps) {
+  // a block takes 16 consecutive features at a time: contiguous gate rows and up rows
+  for (int task = blockIdx.x * (kGuThreads / 32) + warp; task < total; task += nwarps) {
     const int s = task >= f ? 1 : 0;
     const int j = task - s * f;
     const int q = j / kInterleave, i = j % kInterleave;
@@ -162,32 +161,17 @@ gemv_down_combine_kernel(const bf16* __restrict__ act, const bf16* __restrict__ 
   const float w0 = wn[0], w1 = wn[1];
   const int nslot = skipped[0] ? 1 : 2;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // the first loads of the warp's first row go out before the activations are staged, so the
-  // weight stream starts one memory round trip after the routing record is read
   const int n_first = blockIdx.x + gridDim.x * warp;
-  const bool prefetched = n_first < h && nvec >= 256;
-  uint4 pre[8];
-  if (prefetched) {
-    const uint4* w = reinterpret_cast<const uint4*>(W2 + ((size_t)c0 * h + n_first) * f);
-#pragma unroll
-    for (int k = 0; k < 8; ++k) pre[k] = ld_stream(w + lane + 32 * k);
-  }
   for (int v = threadIdx.x; v < nslot * nvec; v += kDnThreads)
     s_act[v] = __ldg(reinterpret_cast<const uint4*>(act) + v);
   __syncthreads();
-  float acc_first = 0.f;
-  if (prefetched) {
-#pragma unroll
-    for (int k = 0; k < 8; ++k) acc_first = dot8(s_act[lane + 32 * k], pre[k], acc_first);
-  }
   for (int n = n_first; n < h; n += gridDim.x * (kDnThreads / 32)) {
     float o0 = 0.f, o1 = 0.f;
     for (int s = 0; s < nslot; ++s) {
       const uint4* w = reinterpret_cast<const uint4*>(W2 + ((size_t)(s ? c1 : c0) * h + n) * f);
       const uint4* av = s_act + s * nvec;
-      const bool first = prefetched && s == 0 && n == n_first;
-      float acc = first ? acc_first : 0.f;
-      int v = first ? lane + 256 : lane;
+      float acc = 0.f;
+      int v = lane;
       for (; v + 224 < nvec; v += 256) {
         uint4 wv[8];
 #pragma unroll
