@@ -299,8 +299,8 @@ def run_ours(a):
 
     if a.workload == "search":
         def step():
-            layer.prune_search(x, 6)
-            layer.prune_search(x, 4)
+            # both subset sizes over one evaluation of the experts (moe_prune_search_multi)
+            layer.prune_search_multi(x, [6, 4])
         launches_per_step = None
     else:
         def step():
@@ -424,9 +424,9 @@ def run_ours(a):
                                         "frac": dn_flop / (dn_ms * 1e-3) / 1e12 / peaks["tf_sust"]},
                         "whole_step_frac": (gu_flop + dn_flop) / (ms_step * 1e-3) / 1e12 / peaks["tf_sust"]}
     elif a.workload == "search":
-        # two searches (r = 6, r = 4); each evaluates a token's E - r + 2 top-ranked experts
+        # r = 6 and r = 4 share one evaluation of each token's E - 4 + 2 = 6 top-ranked experts
         dense = os.environ.get("MOE_SEARCH_DENSE", "") == "1"
-        flop = sum(6 * T * (E if dense else E - r_ + 2) * H * F for r_ in (6, 4))
+        flop = 6 * T * (E if dense else E - 4 + 2) * H * F
         ach = flop / (ms_step * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel (expert evaluations of the search, whole step)",
                     "achieved": ach, "peak": peaks["tf_sust"], "unit": "TFLOP/s",
@@ -455,8 +455,7 @@ def run_ours(a):
         from itertools import combinations
         counts = layer.coselection(x)
         baselines = {}
-        for r_ in (6, 4):
-            losses, best = layer.prune_search(x, r_)
+        for r_, (losses, best) in zip((6, 4), layer.prune_search_multi(x, [6, 4])):
             masks = [sum(1 << i for i in c) for c in combinations(range(E), r_)]
             fmask = layer.frequency_subset(counts, r_)
             baselines["r%d" % r_] = {"searched_subset": best, "searched_loss": min(losses),
@@ -474,7 +473,8 @@ def run_ours(a):
         gpu_launches = launches_per_step * a.steps if launches_per_step else None
         if a.workload == "search":
             chunks = (T + 8191) // 8192
-            gpu_launches = a.steps * 2 * (chunks * 7 + 2)  # per chunk: route, count, scan, scatter, gather, 2 GEMMs
+            # per chunk: route, count, scan, scatter, gather, 2 GEMMs; then enumerate + reduce per size
+            gpu_launches = a.steps * (chunks * 7 + 2 * 2)
         line = {
             "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": a.steps,
             "warmup": max(a.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,

@@ -196,6 +196,19 @@ int moe_calibrate_beta_noalloc(const void* W_gate_kept, const void* x, int T, in
                                void* cuda_stream, float* beta_out);
 
 /*
+ * The same search for several subset sizes r_list[0..n_r-1] at once (Sec. 3.2:
+ * the cached layer inputs and the experts' outputs on them do not depend on r,
+ * only the enumeration does): the experts are evaluated once, for the smallest
+ * size, and every size is enumerated over those outputs.  losses (host) receives
+ * the C(E, r_list[0]) values of the first size, then those of the second, and so
+ * on, each block in the order moe_prune_search uses; best_subsets (host) one
+ * bitmask per size.  Results equal those of one moe_prune_search call per size.
+ * 1 <= n_r <= 16; everything else as moe_prune_search.
+ */
+int moe_prune_search_multi(moe_layer_t* layer, const void* x_calib, int T, const int* r_list,
+                           int n_r, float* losses, uint32_t* best_subsets);
+
+/*
  * Progressive variant of the search (the paper's ablation of layer-wise vs
  * progressive pruning, Sec. 4.4 "Ablation"): the pruned layer is evaluated on
  * x_pruned, calibration states that already went through the pruned earlier

@@ -62,6 +62,8 @@ def load_library(path: str | None = None):
     lib.moe_routing_stats_bytes.argtypes = [ci, ci]
     lib.moe_calibrate_beta.argtypes = [vp, vp, ci, ctypes.POINTER(cf)]
     lib.moe_prune_search.argtypes = [vp, vp, ci, ci, ctypes.POINTER(cf), ctypes.POINTER(u32)]
+    lib.moe_prune_search_multi.argtypes = [vp, vp, ci, ctypes.POINTER(ci), ci, ctypes.POINTER(cf),
+                                           ctypes.POINTER(u32)]
     lib.moe_prune_search_progressive.argtypes = [vp, vp, vp, ci, ci, ctypes.POINTER(cf), ctypes.POINTER(u32)]
     lib.moe_num_subsets.restype = ctypes.c_long
     lib.moe_num_subsets.argtypes = [ci, ci]
@@ -235,6 +237,24 @@ class MoeLayer:
         best = ctypes.c_uint32(0)
         _check(load_library().moe_prune_search(self._h, x_calib.data_ptr(), T, r, losses, ctypes.byref(best)))
         return list(losses)[:n], int(best.value)
+
+    def prune_search_multi(self, x_calib, rs):
+        """``moe_prune_search_multi``: one evaluation of the experts, one enumeration per subset
+        size in ``rs``; returns a list of (losses, best_subset) in the order of ``rs``."""
+        T = x_calib.shape[0]
+        _dev_bf16(x_calib, (T, self.h))
+        rs = [int(r) for r in rs]
+        ns = [comb(self.E, r) if 0 <= r <= self.E else 1 for r in rs]
+        losses = (ctypes.c_float * max(sum(ns), 1))()
+        best = (ctypes.c_uint32 * max(len(rs), 1))()
+        r_arr = (ctypes.c_int * max(len(rs), 1))(*rs)
+        _check(load_library().moe_prune_search_multi(self._h, x_calib.data_ptr(), T, r_arr, len(rs),
+                                                     losses, best))
+        out, o = [], 0
+        for i, n in enumerate(ns):
+            out.append((list(losses[o:o + n]), int(best[i])))
+            o += n
+        return out
 
     def coselection(self, x):
         """``moe_coselection``: E x E list of lists, counts[a][b] = tokens with top-2 (a, b)."""

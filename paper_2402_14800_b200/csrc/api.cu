@@ -660,8 +660,29 @@ uint32_t moe_frequency_subset(const int32_t* counts, int E, int r) {
   return mask;
 }
 
-static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, int T, int r,
-                       float* losses, uint32_t* best_subset) {
+// Subsets of r of E experts in lexicographic order of their ascending index tuples.
+static std::vector<uint32_t> subset_masks(int E, int r) {
+  std::vector<uint32_t> masks;
+  masks.reserve(binom(E, r));
+  int c[kMaxE];
+  for (int i = 0; i < r; ++i) c[i] = i;
+  for (;;) {
+    uint32_t m = 0;
+    for (int i = 0; i < r; ++i) m |= 1u << c[i];
+    masks.push_back(m);
+    int i = r - 1;
+    while (i >= 0 && c[i] == E - r + i) --i;
+    if (i < 0) break;
+    ++c[i];
+    for (int j = i + 1; j < r; ++j) c[j] = c[j - 1] + 1;
+  }
+  return masks;
+}
+
+// The search for n_r subset sizes rs[] over one evaluation of the experts: losses holds the
+// C(E, rs[0]) + C(E, rs[1]) + ... values one after the other, best_subset one mask per size.
+static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, int T, const int* rs,
+                       int n_r, float* losses, uint32_t* best_subset) {
   if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
   if (!x_calib || !losses || !best_subset)
     return fail(MOE_ERR_INVALID_ARG, "x_calib, losses or best_subset is NULL");
@@ -670,35 +691,28 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
     return fail(MOE_ERR_INVALID_ARG, "T = %d outside 1..%d calibration tokens", T, kMaxTokens);
   if (L->r != L->E)
     return fail(MOE_ERR_INVALID_ARG, "the search needs a layer created with all %d experts kept", L->E);
-  if (r < 2 || r > L->E) return fail(MOE_ERR_INVALID_ARG, "r = %d outside 2..%d", r, L->E);
+  if (!rs || n_r < 1 || n_r > kMaxE) return fail(MOE_ERR_INVALID_ARG, "no subset sizes given (or more than %d)", kMaxE);
+  int r = L->E;  // the smallest size: it needs the most experts evaluated per token
+  long nC = 0;   // the largest number of subsets of any size
+  for (int i = 0; i < n_r; ++i) {
+    if (rs[i] < 2 || rs[i] > L->E) return fail(MOE_ERR_INVALID_ARG, "r = %d outside 2..%d", rs[i], L->E);
+    if (rs[i] < r) r = rs[i];
+    if (binom(L->E, rs[i]) > nC) nC = binom(L->E, rs[i]);
+  }
   const int E = L->E, h = L->h, f = L->f;
-  const long nC = binom(E, r);
   cudaStream_t st = L->stream;
   int rc;
   if ((rc = ensure_route(L, T))) return rc;
 
-  // subsets in lexicographic order of their ascending index tuples
-  std::vector<uint32_t> masks;
-  masks.reserve(nC);
-  {
-    int c[kMaxE];
-    for (int i = 0; i < r; ++i) c[i] = i;
-    for (;;) {
-      uint32_t m = 0;
-      for (int i = 0; i < r; ++i) m |= 1u << c[i];
-      masks.push_back(m);
-      int i = r - 1;
-      while (i >= 0 && c[i] == E - r + i) --i;
-      if (i < 0) break;
-      ++c[i];
-      for (int j = i + 1; j < r; ++j) c[j] = c[j - 1] + 1;
-    }
-  }
-
   const int Tc = T < 8192 ? T : 8192;  // tokens per chunk of expert evaluations
   const int Tc_pad = (int)align_up((size_t)Tc, kTileRows);
   const int nchunks = (T + Tc - 1) / Tc;
-  const int nblk_enum = enumerate_num_blocks(T, (int)nC);
+  size_t partial_floats = 0;  // per-block partial losses of the largest enumeration
+  for (int i = 0; i < n_r; ++i) {
+    const size_t n = (size_t)binom(E, rs[i]);
+    const size_t need = (size_t)enumerate_num_blocks(T, (int)n) * n;
+    if (need > partial_floats) partial_floats = need;
+  }
   // A subset of r experts always contains two of a token's K = E - r + 2 top-ranked experts,
   // so only those K need to be evaluated per token (all of them when K = E).
   const int K = E - r + 2;
@@ -706,15 +720,14 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
   Workspace& W = *L->ws;
   if ((rc = grow(L, W.s_logits, (size_t)T * E * 4))) return rc;
   if ((rc = grow(L, W.s_subsets, (size_t)nC * 4))) return rc;
-  if ((rc = grow(L, W.s_partial, (size_t)nblk_enum * nC * 4))) return rc;
+  if ((rc = grow(L, W.s_partial, partial_floats * 4))) return rc;
   if ((rc = grow(L, W.s_loss_sq, (size_t)nC * 8))) return rc;
   if ((rc = grow(L, W.s_losses, (size_t)nC * 4))) return rc;
   if ((rc = grow(L, W.s_meta, sizeof(Meta)))) return rc;
-  CUDA_TRY(cudaMemcpyAsync(W.s_subsets.p, masks.data(), (size_t)nC * 4, cudaMemcpyHostToDevice, st));
   Meta* meta = (Meta*)W.s_meta.p;
   const bool prof_saved = L->prof;
   L->prof = false;  // stage marks describe moe_forward only
-  EnumSource src = {nullptr, nullptr, 0, 0};
+  EnumSource src = {nullptr, nullptr, 0, 0, 0};
   GemmMaps m_gu, m_dn;
   m_gu.w = gemm_pair_mode() ? L->w13_128 : L->w13_256;
   m_dn.w = gemm_pair_mode() ? L->w2_128 : L->w2_256;
@@ -773,6 +786,7 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
     src.pair_pos = (const int32_t*)W.k_pos.p;
     src.chunk_tokens = Tc;
     src.chunk_rows = rows_chunk;
+    src.k_stride = K;
   } else {
     if ((rc = grow(L, W.s_yall, (size_t)T * E * h * 2))) return rc;
     if ((rc = grow(L, W.s_act, ((size_t)E * Tc_pad + kTileRows) * f * 2))) return rc;
@@ -811,28 +825,47 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
     }
   }
   L->prof = prof_saved;
-  CUDA_TRY(launch_enumerate((const float*)W.s_logits.p, (const bf16*)W.s_yall.p, T, E, r, h,
-                            (const uint32_t*)W.s_subsets.p, (int)nC, (float*)W.s_partial.p,
-                            (double*)W.s_loss_sq.p, (float*)W.s_losses.p, F_ref, src, st));
-  CUDA_TRY(cudaMemcpyAsync(losses, L->ws->s_losses.p, (size_t)nC * 4, cudaMemcpyDeviceToHost, st));
+  // one enumeration per subset size over the same expert outputs
+  std::vector<std::vector<uint32_t>> masks(n_r);
+  size_t o = 0;
+  for (int i = 0; i < n_r; ++i) {
+    masks[i] = subset_masks(E, rs[i]);
+    const size_t n = masks[i].size();
+    CUDA_TRY(cudaMemcpyAsync(W.s_subsets.p, masks[i].data(), n * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(launch_enumerate((const float*)W.s_logits.p, (const bf16*)W.s_yall.p, T, E, rs[i], h,
+                              (const uint32_t*)W.s_subsets.p, (int)n, (float*)W.s_partial.p,
+                              (double*)W.s_loss_sq.p, (float*)W.s_losses.p, F_ref, src, st));
+    CUDA_TRY(cudaMemcpyAsync(losses + o, L->ws->s_losses.p, n * 4, cudaMemcpyDeviceToHost, st));
+    o += n;
+  }
   if ((rc = check_status(L))) return rc;
-  long best = 0;
-  for (long c = 1; c < nC; ++c)
-    if (losses[c] < losses[best]) best = c;
-  *best_subset = masks[best];
+  o = 0;
+  for (int i = 0; i < n_r; ++i) {
+    const size_t n = masks[i].size();
+    size_t best = 0;
+    for (size_t c = 1; c < n; ++c)
+      if (losses[o + c] < losses[o + best]) best = c;
+    best_subset[i] = masks[i][best];
+    o += n;
+  }
   return MOE_OK;
 }
 
 int moe_prune_search(moe_layer_t* L, const void* x_calib, int T, int r, float* losses,
                      uint32_t* best_subset) {
-  return search_impl(L, x_calib, nullptr, T, r, losses, best_subset);
+  return search_impl(L, x_calib, nullptr, T, &r, 1, losses, best_subset);
+}
+
+int moe_prune_search_multi(moe_layer_t* L, const void* x_calib, int T, const int* r_list, int n_r,
+                           float* losses, uint32_t* best_subsets) {
+  return search_impl(L, x_calib, nullptr, T, r_list, n_r, losses, best_subsets);
 }
 
 int moe_prune_search_progressive(moe_layer_t* L, const void* x_pruned, const float* F_ref, int T,
                                  int r, float* losses, uint32_t* best_subset) {
   if (!F_ref) return fail(MOE_ERR_INVALID_ARG, "F_ref is NULL");
   if (!aligned16(F_ref)) return fail(MOE_ERR_INVALID_ARG, "F_ref must be 16-byte aligned");
-  return search_impl(L, x_pruned, F_ref, T, r, losses, best_subset);
+  return search_impl(L, x_pruned, F_ref, T, &r, 1, losses, best_subset);
 }
 
 int moe_rmsnorm(const void* x, int T, int h, float eps, void* out, void* cuda_stream) {

@@ -231,6 +231,7 @@ struct EnumSource {
   const int32_t* pair_pos;
   int chunk_tokens;
   int chunk_rows;
+  int k_stride;  // ranked experts recorded per token in topk_idx / pair_pos (>= E - r + 2)
 };
 int enumerate_num_blocks(int T, int nC);
 cudaError_t launch_enumerate(const float* logits, const bf16* Yall, int T, int E, int r, int h,

@@ -160,8 +160,8 @@ enumerate_kernel(const float* __restrict__ logits, const bf16* __restrict__ Yall
       // only the K top-ranked experts were evaluated; they are listed in rank order, and their
       // outputs sit in the permuted row pair_pos[t][rank] of the token's chunk
       if (lane < K) {
-        s_order[lane] = src.topk_idx[(size_t)t * K + lane];
-        s_row[lane] = (t / src.chunk_tokens) * src.chunk_rows + src.pair_pos[(size_t)t * K + lane];
+        s_order[lane] = src.topk_idx[(size_t)t * src.k_stride + lane];
+        s_row[lane] = (t / src.chunk_tokens) * src.chunk_rows + src.pair_pos[(size_t)t * src.k_stride + lane];
       }
     } else if (lane < E) {
       int rank = 0;

@@ -64,6 +64,7 @@ def test_create_rejects_bad_arguments_without_a_device(lib):
 def test_null_handle_is_an_error(lib):
     assert lib.moe_forward(None, None, 4, 0.0, None, None) == -1
     assert lib.moe_prune_search(None, None, 4, 6, None, None) == -1
+    assert lib.moe_prune_search_multi(None, None, 4, None, 2, None, None) == -1
     assert lib.moe_calibrate_beta(None, None, 4, None) == -1
     assert lib.moe_device_status(None) == -1
     assert lib.moe_layer_weight_bytes(None) == 0

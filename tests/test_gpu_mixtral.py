@@ -129,6 +129,11 @@ def test_search_full_size_invariants(big):
     np.testing.assert_allclose(np.square(a) + np.square(b), np.square(whole), rtol=1e-4)
     full, bestf = layer.prune_search(x[:4096].contiguous(), 8)
     assert full == [0.0] and bestf == FULL
+    # both configured sizes over one evaluation of the experts (what bench.py times)
+    (l6, b6), (l4, b4) = layer.prune_search_multi(x, [6, 4])
+    assert l6 == whole and b6 == best
+    l4s, b4s = layer.prune_search(x, 4)
+    assert l4 == l4s and b4 == b4s and len(l4) == 70
     # the loss of a subset is carried by the tokens whose top-2 it breaks: more broken tokens, on
     # average, more loss -- checked through the routing record of the same batch
     stats = binding.RoutingStats(T, E, DEV)

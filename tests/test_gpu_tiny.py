@@ -181,6 +181,29 @@ def test_calibrate_beta(setup, T):
     assert abs(got - want) <= 2e-6 * max(1.0, abs(want))
 
 
+@pytest.mark.parametrize("T", [256, 700])
+def test_prune_search_multi_equals_one_search_per_size(setup, T):
+    # several subset sizes over one evaluation of the experts: same losses, same argmin as a
+    # separate search per size, and the oracle's
+    host, dev = setup
+    x = synth.make_tokens(T, H, seed=5)
+    layer = make_layer(dev)
+    rs = [6, 4, 7, 8]
+    multi = layer.prune_search_multi(x.to(DEV), rs)
+    for r, (losses, best) in zip(rs, multi):
+        single, best1 = layer.prune_search(x.to(DEV), r)
+        assert losses == single and best == best1
+    ora = O.prune_search_allexperts(synth.bf16_bits(x), host["Wg"], host["W1"], host["W3"], host["W2"], 4)
+    P.check_search(multi[1][0], multi[1][1], ora)
+    one = layer.prune_search_multi(x.to(DEV), [5])
+    assert one[0] == tuple(layer.prune_search(x.to(DEV), 5))
+    with pytest.raises(binding.MoeError):
+        layer.prune_search_multi(x.to(DEV), [6, 1])
+    with pytest.raises(binding.MoeError):
+        layer.prune_search_multi(x.to(DEV), [])
+    layer.close()
+
+
 @pytest.mark.parametrize("r", [6, 4, 8, 2])
 def test_prune_search_matches_oracle(setup, r):
     host, dev = setup
