@@ -398,7 +398,7 @@ def run_ours(a):
             forced = os.environ.get("MOE_DECODE_KERNEL", "")
             r_kept = bin(KEPT[a.kept]).count("1")
             # the library's crossover: many tokens per expert -> token-major decode kernel
-            token_major = forced == "td" or (forced != "wm" and 2 * a.tokens >= 40 * r_kept)
+            token_major = forced == "td" or (forced != "wm" and 2 * a.tokens >= 40 * r_kept and r_kept <= 6)
             kernel = "gemm_tokens_d_kernel<gate_up>" if token_major else "gemm_weights_m_kernel<gate_up>"
             if single_gemv:  # one token: matrix-vector kernels on the CUDA cores
                 kernel = "gemv_route_gate_up_kernel"

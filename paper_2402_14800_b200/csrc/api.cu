@@ -99,6 +99,7 @@ struct moe_layer {
   bool prof = false;
   std::vector<cudaEvent_t> prof_ev;  // MOE_PROFILE_STAGES + 1 marks per recorded call
   size_t prof_used = 0;
+  int* h_status = nullptr;  // pinned host copy of the device status word
 };
 
 namespace {
@@ -156,9 +157,12 @@ int ensure_route(moe_layer* L, int T) {
 
 inline bool decode_mode(int T) { return T <= kDecodeMaxT; }
 // Small batches run the weight-major GEMM unless the experts hold many tokens each (about
-// 2T/r): from kTokensDPerExpert on, the token-major decode GEMM is faster (measured crossover).
+// 2T/r): from kTokensDPerExpert on, the token-major decode GEMM is faster on layers of at most
+// kTokensDMaxKept kept experts (measured crossover; with 8 experts the weight-major kernel won
+// up to the largest small batch, 64 tokens per expert).
 inline bool decode_weights_m(const moe_layer* L, int T) {
-  return L->decode_kernel == 1 || (L->decode_kernel == 0 && 2 * T < kTokensDPerExpert * L->r);
+  return L->decode_kernel == 1 ||
+         (L->decode_kernel == 0 && (2 * T < kTokensDPerExpert * L->r || L->r > kTokensDMaxKept));
 }
 inline int rows_for(const moe_layer* L, int T, int k = 2) {
   const int pad = decode_mode(T) ? 16 : kTileRows;
@@ -221,9 +225,16 @@ void mark(moe_layer* L) {
 }
 
 int check_status(moe_layer* L) {
-  int st = 0;
-  CUDA_TRY(cudaMemcpyAsync(&st, L->ws->status.p, 4, cudaMemcpyDeviceToHost, L->stream));
+  // the status word is read into pinned memory: a copy to pageable memory is staged by the runtime
+  if (!L->h_status && cudaHostAlloc((void**)&L->h_status, sizeof(int), cudaHostAllocDefault) != cudaSuccess) {
+    cudaGetLastError();
+    L->h_status = nullptr;
+  }
+  int st_pageable = 0;
+  int* dst = L->h_status ? L->h_status : &st_pageable;
+  CUDA_TRY(cudaMemcpyAsync(dst, L->ws->status.p, 4, cudaMemcpyDeviceToHost, L->stream));
   CUDA_TRY(cudaStreamSynchronize(L->stream));
+  const int st = *dst;
   if (st != 0) {
     cudaMemsetAsync(L->ws->status.p, 0, 4, L->stream);
     // an aborted GEMM may have left arrival counters of its K-sliced tail items behind
@@ -493,6 +504,7 @@ void moe_layer_destroy(moe_layer_t* L) {
                  &L->own.s_losses, &L->own.s_xpad, &L->own.s_meta, &L->own.s_xperm, &L->own.s_rowtok, &L->own.hx, &L->own.hy, &L->own.xn, &L->own.cosel, &L->own.k_idx, &L->own.k_wn, &L->own.k_pos, &L->own.k_nact};
   for (Buf* b : bufs) release(L, *b);
   for (cudaEvent_t e : L->prof_ev) cudaEventDestroy(e);
+  if (L->h_status) cudaFreeHost(L->h_status);
   if (L->Wg) cudaFree(L->Wg);
   if (L->W13) cudaFree(L->W13);
   if (L->W2) cudaFree(L->W2);

@@ -19,6 +19,7 @@ constexpr int kHistCols = 2 * kMaxE + 1;  // per (expert, slot) pair counts + sk
 constexpr int kInterleave = 16;           // W1/W3 rows are interleaved in groups of 16
 constexpr int kDecodeMaxT = 256;          // up to here the small-batch path (weights read once) is used
 constexpr int kTokensDPerExpert = 40;      // small batches with this many tokens per expert or more: token-major decode GEMM
+constexpr int kTokensDMaxKept = 6;         // ... on layers with at most this many kept experts
 #ifndef MOE_DOWN_KB
 #define MOE_DOWN_KB 112
 #endif
