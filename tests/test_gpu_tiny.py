@@ -262,6 +262,31 @@ def test_rmsnorm_and_stack(setup):
         l.close()
 
 
+def test_stack_of_single_tokens(setup):
+    # batch-1 decoding through three layers (RMSNorm, single-token kernels with the residual)
+    specs = [(20, FULL, 0.0), (21, 0b10111011, 0.4), (22, 0b00111100, 0.5)]
+    b = synth.bf16_bits
+    Ws = [synth.make_layer_weights(H, F, E, seed=seed) for seed, _, _ in specs]
+    layers = [binding.MoeLayer(W.W_gate.to(DEV), W.W1.to(DEV), W.W3.to(DEV), W.W2.to(DEV), kept)
+              for W, (_, kept, _) in zip(Ws, specs)]
+    errs = []
+    for seed in range(8):
+        x = synth.make_tokens(1, H, seed=60 + seed)
+        cur = b(x)
+        for W, (_, kept, beta) in zip(Ws, specs):
+            xn = O.rmsnorm(cur, 1e-5)
+            cur = O.moe_forward(xn, b(W.W_gate), b(W.W1), b(W.W3), b(W.W2), kept, beta, residual=cur)["y"]
+        y = binding.stack_forward(layers, x.to(DEV), [s[2] for s in specs], 1e-5)
+        torch.cuda.synchronize()
+        g, o = P.bf16_bits_to_f64(b(y)), P.bf16_bits_to_f64(cur)
+        errs.append(float(np.linalg.norm(g - o) / np.linalg.norm(o)))
+    # a token re-routed by a near-tie in an early layer may differ; the others obey the bound
+    assert sorted(errs)[-2] <= P.Y_REL_L2_TOL, errs
+    for l in layers:
+        assert l.device_status() == 0
+        l.close()
+
+
 @pytest.mark.parametrize("h,f,E,kept,T", [
     (192, 320, 4, 0b1111, 300),     # ragged K and N tiles, few experts
     (192, 320, 4, 0b1011, 40),
