@@ -298,6 +298,9 @@ constexpr int TM_A_BYTES = 128 * 128;  // 128 token rows x 64 bf16
 constexpr int TM_B_BYTES = 256 * 128;  // 256 weight rows x 64 bf16
 constexpr int TM_STAGE = TM_A_BYTES + TM_B_BYTES;
 constexpr int TM_SMEM = TM_NS * TM_STAGE + 1024;
+#ifndef MOE_TM_KB_PAIRS
+#define MOE_TM_KB_PAIRS 1  // MMA issuer of the token-major kernel: two k-blocks per loop trip (0: one)
+#endif
 constexpr int TM_BN = 256;
 
 // Epilogue of one 128-row x 256-column accumulator tile of the token-major kernels: this
@@ -414,7 +417,36 @@ gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args)
       if (!ok) break;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + buf * TM_BN;
-      for (int kb = 0; kb < KB; ++kb, ++it) {
+      int kb = 0;
+#if MOE_TM_KB_PAIRS
+      // two k-blocks per trip round the loop: both stages are awaited, then one fence, eight
+      // MMAs, and the commit of each stage right after its own four
+      for (; kb + 1 < KB; kb += 2, it += 2) {
+        const uint32_t s0 = it % TM_NS, ph0 = (it / TM_NS) & 1u;
+        const uint32_t s1 = (it + 1) % TM_NS, ph1 = ((it + 1) / TM_NS) & 1u;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[s0]), ph0, abort_flag) &&
+                                         mbar_wait(smem_u32(&bars.full[s1]), ph1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t sa0 = smem_base + s0 * TM_STAGE, sa1 = smem_base + s1 * TM_STAGE;
+          const uint64_t adesc0 = smem_desc_k128(sa0), bdesc0 = smem_desc_k128(sa0 + TM_A_BYTES);
+          const uint64_t adesc1 = smem_desc_k128(sa1), bdesc1 = smem_desc_k128(sa1 + TM_A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_bf16(d_tmem, adesc0 + 2 * k, bdesc0 + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(smem_u32(&bars.empty[s0]));
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_bf16(d_tmem, adesc1 + 2 * k, bdesc1 + 2 * k, idesc, 1u);
+          umma_commit(smem_u32(&bars.empty[s1]));
+          if (kb + 2 == KB) umma_commit(smem_u32(&bars.tmem_full[buf]));
+        }
+        __syncwarp();
+      }
+      if (!ok) break;
+#endif
+      for (; kb < KB; ++kb, ++it) {
         const uint32_t s = it % TM_NS, ph = (it / TM_NS) & 1u;
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag));
         if (!ok) break;

@@ -33,6 +33,19 @@ __device__ __forceinline__ float dot8(const uint4& a, const uint4& w, float acc)
 // activations and the routing record.
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 
+// Whatever an earlier kernel of the stream wrote (the token row, the activations, the routing
+// record, the residual) is read at L2 (ld.global.cg).  These kernels start as programmatic
+// dependents while their predecessor still runs, so their lifetime overlaps the writer's: the
+// non-coherent path (ld.global.nc) is only for data that never changes, and an L1 line cached
+// on this SM before the writer finished would be stale.
+__device__ __forceinline__ uint4 ld_l2(const uint4* p) { return __ldcg(p); }
+__device__ __forceinline__ int ld_l2(const int32_t* p) { return __ldcg(p); }
+__device__ __forceinline__ float ld_l2(const float* p) { return __ldcg(p); }
+__device__ __forceinline__ int ld_l2(const uint8_t* p) { return (int)__ldcg(p); }
+__device__ __forceinline__ float ld_l2(const bf16* p) {
+  return __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p)) << 16);
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
@@ -71,7 +84,7 @@ gemv_route_gate_up_kernel(const bf16* __restrict__ x, const bf16* __restrict__ W
 #pragma unroll
   for (int c = 0; c < R; ++c) acc[c] = 0.f;
   for (int v = threadIdx.x; v < nvec; v += kGuThreads) {
-    const uint4 xv = __ldg(reinterpret_cast<const uint4*>(x) + v);
+    const uint4 xv = ld_l2(reinterpret_cast<const uint4*>(x) + v);
     s_x[v] = xv;
     constexpr int G = R < 8 ? R : 8;  // router rows fetched together
 #pragma unroll
@@ -79,7 +92,7 @@ gemv_route_gate_up_kernel(const bf16* __restrict__ x, const bf16* __restrict__ W
       uint4 wv[G];
 #pragma unroll
       for (int c = 0; c < G; ++c)
-        if (cb + c < r) wv[c] = __ldg(reinterpret_cast<const uint4*>(Wg + (size_t)(cb + c) * h) + v);
+        if (cb + c < r) wv[c] = ld_l2(reinterpret_cast<const uint4*>(Wg + (size_t)(cb + c) * h) + v);
 #pragma unroll
       for (int c = 0; c < G; ++c)
         if (cb + c < r) acc[cb + c] = dot8(xv, wv[c], acc[cb + c]);
@@ -157,13 +170,13 @@ gemv_down_combine_kernel(const bf16* __restrict__ act, const bf16* __restrict__ 
   pdl_launch_dependents();
   pdl_wait();
   const int nvec = f >> 3;
-  const int c0 = idx[0], c1 = idx[1];  // compact expert indices of the two slots
-  const float w0 = wn[0], w1 = wn[1];
-  const int nslot = skipped[0] ? 1 : 2;
+  const int c0 = ld_l2(idx), c1 = ld_l2(idx + 1);  // compact expert indices of the two slots
+  const float w0 = ld_l2(wn), w1 = ld_l2(wn + 1);
+  const int nslot = ld_l2(skipped) ? 1 : 2;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int n_first = blockIdx.x + gridDim.x * warp;
   for (int v = threadIdx.x; v < nslot * nvec; v += kDnThreads)
-    s_act[v] = __ldg(reinterpret_cast<const uint4*>(act) + v);
+    s_act[v] = ld_l2(reinterpret_cast<const uint4*>(act) + v);
   __syncthreads();
   for (int n = n_first; n < h; n += gridDim.x * (kDnThreads / 32)) {
     float o0 = 0.f, o1 = 0.f;
@@ -185,7 +198,7 @@ gemv_down_combine_kernel(const bf16* __restrict__ act, const bf16* __restrict__ 
     }
     if (lane == 0) {
       float z = (nslot == 2) ? fmaf(w1, o1, w0 * o0) : w0 * o0;
-      if (residual) z += __bfloat162float(residual[n]);
+      if (residual) z += ld_l2(residual + n);
       y[n] = __float2bfloat16_rn(z);
     }
   }
