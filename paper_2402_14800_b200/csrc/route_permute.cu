@@ -6,6 +6,11 @@
 //                   no atomics, the order is a function of the routing alone.
 //   gather          copies the routed rows of x into expert-contiguous order.
 //   combine         Eq. 2: y = bf16(residual + w~_e0 o_e0 + w~_e1 o_e1), slot 0 first.
+//
+// The token rows (x) are read with ld.global.cg (L2), not through the non-coherent path: in a
+// stack the kernel that wrote them (RMSNorm, the previous layer's combine) may still be running
+// when these kernels start as its programmatic dependents, and an L1 line cached before the
+// writer finished would be stale.  The router rows never change and keep ld.global.nc.
 #include "common.h"
 #include "route_device.cuh"
 
@@ -31,7 +36,7 @@ router_small_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
   const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)t * h);
   for (int v = threadIdx.x; v < nvec; v += 256) {
     float xf[8];
-    unpack8(__ldg(xr + v), xf);
+    unpack8(__ldcg(xr + v), xf);
 #pragma unroll
     for (int c = 0; c < R; ++c) {
       if (c < r) {
@@ -85,7 +90,7 @@ route_single_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
   const uint4* xr = reinterpret_cast<const uint4*>(x);
   for (int v = threadIdx.x; v < nvec; v += 256) {
     float xf[8];
-    unpack8(__ldg(xr + v), xf);
+    unpack8(__ldcg(xr + v), xf);
 #pragma unroll
     for (int c = 0; c < R; ++c) {
       if (c < r) {
@@ -124,7 +129,7 @@ route_single_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
   uint4* d0 = reinterpret_cast<uint4*>(xperm + (size_t)p0 * h);
   uint4* d1 = reinterpret_cast<uint4*>(xperm + (size_t)(p1 < 0 ? p0 : p1) * h);
   for (int v = threadIdx.x; v < nvec; v += 256) {
-    const uint4 val = __ldg(xr + v);
+    const uint4 val = __ldcg(xr + v);
     d0[v] = val;
     if (p1 >= 0) d1[v] = val;
   }
@@ -227,7 +232,7 @@ permute_gather_small_kernel(const bf16* __restrict__ x, const int32_t* __restric
   uint4* d0 = reinterpret_cast<uint4*>(xperm + (size_t)p0 * h);
   uint4* d1 = reinterpret_cast<uint4*>(xperm + (size_t)(p1 < 0 ? p0 : p1) * h);
   for (int v = i; v < nvec; v += blockDim.x) {
-    const uint4 val = __ldg(src + v);
+    const uint4 val = __ldcg(src + v);
     d0[v] = val;
     if (p1 >= 0) d1[v] = val;
   }
@@ -260,7 +265,7 @@ router_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, in
     uint4 xv[kRouteXVec];
 #pragma unroll
     for (int i = 0; i < kRouteXVec; ++i)
-      xv[i] = (v0 + 32 * i < nvec) ? __ldg(xr + v0 + 32 * i) : make_uint4(0u, 0u, 0u, 0u);
+      xv[i] = (v0 + 32 * i < nvec) ? __ldcg(xr + v0 + 32 * i) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
     for (int i = 0; i < kRouteXVec; ++i) {
       const int v = v0 + 32 * i;
@@ -439,7 +444,7 @@ gather_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ row_token,
     uint4* dst = reinterpret_cast<uint4*>(xperm + (size_t)row * h);
     if (t >= 0) {
       const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * h);
-      for (int v = lane; v < nvec; v += 32) dst[v] = __ldg(src + v);
+      for (int v = lane; v < nvec; v += 32) dst[v] = __ldcg(src + v);
     } else {
       for (int v = lane; v < nvec; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
     }
@@ -514,7 +519,7 @@ router_topk_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int 
   const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)t * h);
   for (int v = threadIdx.x; v < nvec; v += 256) {
     float xf[8];
-    unpack8(__ldg(xr + v), xf);
+    unpack8(__ldcg(xr + v), xf);
 #pragma unroll
     for (int c = 0; c < kMaxE; ++c) {
       if (c < r) {
