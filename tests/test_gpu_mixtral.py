@@ -194,3 +194,27 @@ def test_topk_and_progressive_at_full_shape(big):
                                        F_ref.cpu().numpy(), 6)
     losses, best = layer.prune_search_progressive(x, F_ref, 6)
     P.check_search(losses, best, ora_p)
+
+
+@pytest.mark.parametrize("T,kept", [(1, FULL), (8, FULL), (128, FULL), (128, 0x0F), (2048, FULL)])
+def test_back_to_back_steps_with_changing_inputs(big, T, kept):
+    # Serving pattern at full shape: one input buffer refilled every step, the steps queued
+    # without synchronising (their kernels overlap through programmatic dependent launch); each
+    # step must reproduce the isolated call on the same input bit for bit.
+    n = 6
+    layer = big["layer"](kept)
+    xs = [synth.make_tokens(T, H, seed=300 + i, device=DEV) for i in range(n)]
+    want = []
+    for x in xs:
+        want.append(layer.forward(x, 0.3).clone())
+        torch.cuda.synchronize()
+    x_buf = torch.empty_like(xs[0])
+    ys = [torch.empty_like(xs[0]) for _ in range(n)]
+    for rep in range(3):
+        for i in range(n):
+            x_buf.copy_(xs[i])
+            layer.forward(x_buf, 0.3, y=ys[i])
+        torch.cuda.synchronize()
+        for i in range(n):
+            assert torch.equal(ys[i], want[i]), "step %d of round %d differs from the isolated call" % (i, rep)
+    assert layer.device_status() == 0

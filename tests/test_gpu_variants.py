@@ -151,3 +151,28 @@ def test_forward_replays_from_a_cuda_graph(weights, T):
         s.synchronize()
         assert torch.equal(y, fresh)
     layer.close()
+
+
+@pytest.mark.parametrize("T", [1, 2, 8, 40, 128, 600])
+def test_back_to_back_calls_with_changing_inputs_equal_isolated_calls(weights, T):
+    # Serving pattern: the same buffers, new contents every step, the calls queued without a
+    # synchronisation in between (the kernels of consecutive calls overlap through programmatic
+    # dependent launch).  Every step must give what the same input gives in an isolated call.
+    n = 12
+    layer = binding.MoeLayer(*weights, 0b11110111)
+    xs = [synth.make_tokens(T, H, seed=200 + i).to(DEV) for i in range(n)]
+    want = []
+    for x in xs:
+        want.append(layer.forward(x, 0.4).clone())
+        torch.cuda.synchronize()
+    x_buf = torch.empty_like(xs[0])
+    ys = [torch.empty_like(xs[0]) for _ in range(n)]
+    for rep in range(3):
+        for i in range(n):
+            x_buf.copy_(xs[i])
+            layer.forward(x_buf, 0.4, y=ys[i])
+        torch.cuda.synchronize()
+        for i in range(n):
+            assert torch.equal(ys[i], want[i]), "step %d of round %d differs from the isolated call" % (i, rep)
+    assert layer.device_status() == 0
+    layer.close()
