@@ -72,6 +72,17 @@ int moe_set_stream(moe_layer_t* layer, void* cuda_stream);
  */
 int moe_layer_share_scratch(moe_layer_t* layer, moe_layer_t* owner);
 
+/*
+ * Grow the handle's scratch now to what moe_forward / moe_forward_residual need
+ * for any batch of 1 .. T_max tokens (both the small-batch and the large-batch
+ * kernel sequences), so that no later forward call with T <= T_max allocates,
+ * frees or synchronises the device: a serving loop calls this once at start-up,
+ * and a CUDA-graph capture needs no warm-up call.  Not part of the paper's
+ * method.  Synchronises the handle's stream when a buffer is replaced.
+ * Errors: MOE_ERR_INVALID_ARG (T_max outside 1 .. 2^24), MOE_ERR_OOM.
+ */
+int moe_reserve(moe_layer_t* layer, int T_max);
+
 /* Bytes of device memory the handle holds for weights (router + kept experts). */
 size_t moe_layer_weight_bytes(const moe_layer_t* layer);
 
@@ -184,8 +195,12 @@ int moe_prune_search(moe_layer_t* layer, const void* x_calib, int T, int r, floa
  * loading the library holds until the process exits; T is therefore limited to
  * MOE_NOALLOC_MAX_TOKENS and larger T is rejected with MOE_ERR_INVALID_ARG.
  * The call makes no cudaMalloc/cudaFree and calls no allocating library
- * routine.  Its first call on a device looks up the array's device address
- * (cudaGetSymbolAddress); make that first call before any stream capture.
+ * routine.  Its first call on a device is a warm-up: it looks up the array's
+ * device address (cudaGetSymbolAddress), and under CUDA's lazy module loading
+ * that look-up or the first launch may load this part of the library onto the
+ * device, which takes device memory once (the code and the array).  Make that
+ * first call at start-up, before any stream capture and before the device is
+ * handed to the caller's own memory pool; the calls after it take nothing.
  * All calls share the one array, which keeps the previous call's contents:
  * every element that is read is rewritten first, so nothing needs clearing,
  * but two calls that overlap on the GPU (different streams or threads) race.

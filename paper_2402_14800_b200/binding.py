@@ -37,7 +37,7 @@ def load_library(path: str | None = None):
     global _lib
     if _lib is not None and path is None:
         return _lib
-    p = path or os.environ.get("MOE_LIBRARY") or _LIB_PATH  # MOE_LIBRARY: another build of the library
+    p = path or _LIB_PATH
     if not os.path.exists(p):
         raise MoeError(-3, "%s not found: build it with `python -m paper_2402_14800_b200.build`" % p)
     lib = ctypes.CDLL(p)
@@ -77,6 +77,10 @@ def load_library(path: str | None = None):
     lib.moe_profile_enable.argtypes = [vp, ci]
     lib.moe_profile_read.argtypes = [vp, ctypes.POINTER(cf), ctypes.POINTER(ci)]
     lib.moe_calibrate_beta_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, ctypes.POINTER(cf)]
+    lib.moe_reserve.argtypes = [vp, ci]
+    lib.moe_test_wait_expiry.argtypes = [vp, ctypes.c_uint, ci]
+    lib.moe_test_set_free_bytes_limit.restype = None
+    lib.moe_test_set_free_bytes_limit.argtypes = [ctypes.c_longlong]
     lib.moe_last_error.restype = ctypes.c_char_p
     if path is None:
         _lib = lib
@@ -162,6 +166,10 @@ class MoeLayer:
     def share_scratch(self, owner: "MoeLayer | None"):
         """Run out of ``owner``'s scratch buffers (``moe_layer_share_scratch``)."""
         _check(load_library().moe_layer_share_scratch(self._h, owner._h if owner is not None else None))
+
+    def reserve(self, T_max: int):
+        """``moe_reserve``: grow the scratch for any forward batch of up to ``T_max`` tokens now."""
+        _check(load_library().moe_reserve(self._h, int(T_max)))
 
     @property
     def weight_bytes(self) -> int:

@@ -46,26 +46,6 @@ def up_to_date() -> bool:
     return all(os.path.getmtime(d) <= t for d in _deps())
 
 
-def build_variant(lib_path: str, extra_flags) -> str:
-    """Build a copy of the library with extra nvcc flags (for example -DMOE_KBAND=8) under
-    another name, for side-by-side measurements; select it with MOE_LIBRARY=<path>."""
-    import tempfile
-    nvcc = _nvcc()
-    with tempfile.TemporaryDirectory() as tmp:
-        objs = []
-        for src in sources():
-            obj = os.path.join(tmp, os.path.basename(src)[:-3] + ".o")
-            r = subprocess.run([nvcc] + NVCC_FLAGS + list(extra_flags) + ["-c", src, "-o", obj],
-                               capture_output=True, text=True)
-            if r.returncode != 0:
-                raise RuntimeError("nvcc failed for %s:\n%s\n%s" % (src, r.stdout, r.stderr))
-            objs.append(obj)
-        r = subprocess.run([nvcc, "-shared", "-o", lib_path] + objs, capture_output=True, text=True)
-        if r.returncode != 0:
-            raise RuntimeError("link failed:\n%s\n%s" % (r.stdout, r.stderr))
-    return lib_path
-
-
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and up_to_date():
         return LIB

@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "common.h"
+#include "moe_test_hooks.h"
 
 using namespace moe;
 
@@ -41,6 +42,17 @@ long binom(int n, int k) {
   long r = 1;
   for (int i = 1; i <= k; ++i) r = r * (n - k + i) / i;
   return r;
+}
+
+// Test hook (moe_test_set_free_bytes_limit): an upper bound on what cudaMemGetInfo may report.
+long long g_free_bytes_limit = -1;
+
+cudaError_t free_device_bytes(size_t* free_b) {
+  size_t total_b = 0;
+  cudaError_t e = cudaMemGetInfo(free_b, &total_b);
+  if (e == cudaSuccess && g_free_bytes_limit >= 0 && *free_b > (size_t)g_free_bytes_limit)
+    *free_b = (size_t)g_free_bytes_limit;
+  return e;
 }
 
 // A device buffer that only grows.
@@ -113,8 +125,8 @@ int grow(moe_layer* L, Buf& b, size_t bytes) {
     b.p = nullptr;
     b.bytes = 0;
   }
-  size_t free_b = 0, total_b = 0;
-  if (cudaMemGetInfo(&free_b, &total_b) == cudaSuccess && bytes > free_b)
+  size_t free_b = 0;
+  if (free_device_bytes(&free_b) == cudaSuccess && bytes > free_b)
     return fail(MOE_ERR_OOM, "scratch of %zu bytes does not fit (%zu free)", bytes, free_b);
   cudaError_t e = cudaMalloc(&b.p, bytes);
   if (e != cudaSuccess) {
@@ -144,6 +156,8 @@ int ensure_route(moe_layer* L, int T) {
   if ((rc = grow(L, L->ws->sel, 16))) return rc;
   if (T <= L->ws->cap_route_T) return MOE_OK;
   const size_t nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
+  // a buffer that fails to grow is gone: the capacity is void until every buffer has grown
+  L->ws->cap_route_T = 0;
   if ((rc = grow(L, L->ws->idx, (size_t)T * 8))) return rc;
   if ((rc = grow(L, L->ws->wn, (size_t)T * 8))) return rc;
   if ((rc = grow(L, L->ws->ratio, (size_t)T * 4))) return rc;
@@ -193,6 +207,7 @@ int ensure_gemm(moe_layer* L, int T, int k = 2) {
     return MOE_OK;
   if (need < L->ws->cap_rows) need = L->ws->cap_rows;
   int rc;
+  L->ws->cap_rows = 0;  // void until every buffer has grown and the tensor maps are rebuilt
   if ((rc = grow(L, L->ws->row_token, (size_t)need * 4))) return rc;
   if ((rc = grow(L, L->ws->xperm, (size_t)need * L->h * 2))) return rc;
   if ((rc = grow(L, L->ws->act, (size_t)need * L->f * 2))) return rc;
@@ -358,8 +373,8 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;
   GemmMaps m_gu, m_dn;
-  m_gu.w = (wm ? decode_weights_m(L, T) : gemm_pair_mode()) ? L->w13_128 : L->w13_256;
-  m_dn.w = (wm ? decode_weights_m(L, T) : gemm_pair_mode()) ? L->w2_128 : L->w2_256;
+  m_gu.w = (wm && decode_weights_m(L, T)) ? L->w13_128 : L->w13_256;
+  m_dn.w = (wm && decode_weights_m(L, T)) ? L->w2_128 : L->w2_256;
   memcpy(m_gu.t, L->ws->tok_x, sizeof(m_gu.t));
   memcpy(m_dn.t, L->ws->tok_act, sizeof(m_dn.t));
   rc = run_expert_gemms(L, meta, wm, m_gu, m_dn, gu, dn, kOutF32, (const bf16*)L->ws->xperm.p,
@@ -445,15 +460,13 @@ moe_layer_t* moe_layer_create(const void* W_gate, const void* W1, const void* W3
   L->single_gemv = !(sk && !strcmp(sk, "gemm")) && L->decode_kernel == 0 && gemv_single_fits(h, f);
   const char* nopdl = getenv("MOE_NO_PDL");
   if (nopdl) g_pdl_enabled = nopdl[0] != '1';
-  const char* pair = getenv("MOE_GEMM_PAIR");
-  if (pair) gemm_set_pair_mode(pair[0] == '1');
   const char* dense = getenv("MOE_SEARCH_DENSE");
   L->search_dense = dense && dense[0] == '1';
 
   const size_t n_gate = (size_t)L->r * h * 2, n_13 = (size_t)L->r * 2 * f * h * 2,
                n_2 = (size_t)L->r * h * f * 2;
-  size_t free_b = 0, total_b = 0;
-  cudaMemGetInfo(&free_b, &total_b);
+  size_t free_b = 0;
+  if (free_device_bytes(&free_b) != cudaSuccess) free_b = ~(size_t)0;
   if (n_gate + n_13 + n_2 > free_b) {
     fail(MOE_ERR_OOM, "weights of %zu bytes do not fit (%zu free)", n_gate + n_13 + n_2, free_b);
     delete L;
@@ -514,6 +527,33 @@ void moe_layer_destroy(moe_layer_t* L) {
 int moe_set_stream(moe_layer_t* L, void* cuda_stream) {
   if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
   L->stream = (cudaStream_t)cuda_stream;
+  return MOE_OK;
+}
+
+int moe_reserve(moe_layer_t* L, int T_max) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  if (T_max < 1 || T_max > kMaxTokens) return fail(MOE_ERR_INVALID_ARG, "T_max = %d outside 1..%d", T_max, kMaxTokens);
+  int rc;
+  if ((rc = ensure_route(L, T_max))) return rc;
+  // the small-batch sequences want split-K planes, the large-batch ones more rows: take both
+  if ((rc = ensure_gemm(L, T_max < kDecodeMaxT ? T_max : kDecodeMaxT))) return rc;
+  if ((rc = ensure_gemm(L, 1))) return rc;  // one or two tokens use finer split-K items
+  if ((rc = ensure_gemm(L, T_max))) return rc;
+  return MOE_OK;
+}
+
+void moe_test_set_free_bytes_limit(long long bytes) { g_free_bytes_limit = bytes; }
+
+int moe_test_wait_expiry(moe_layer_t* L, unsigned limit_us, int poison_tail) {
+  if (!L) return fail(MOE_ERR_INVALID_ARG, "layer is NULL");
+  if (limit_us < 1 || limit_us > 100000) return fail(MOE_ERR_INVALID_ARG, "limit_us = %u outside 1..100000", limit_us);
+  int rc;
+  if ((rc = ensure_route(L, 1))) return rc;
+  if (poison_tail) {
+    if ((rc = ensure_gemm(L, 1))) return rc;
+    CUDA_TRY(cudaMemsetAsync(L->ws->tail.p, 0x01, 64, L->stream));
+  }
+  CUDA_TRY(launch_wait_expiry((int*)L->ws->status.p, (unsigned long long)limit_us * 1000ull, L->stream));
   return MOE_OK;
 }
 
@@ -581,8 +621,8 @@ int moe_forward_topk(moe_layer_t* L, const void* x, int T, int k, float beta, vo
   const size_t split_stride = (size_t)rows_cap * L->h;
   dn.split_stride = (long long)split_stride;
   GemmMaps m_gu, m_dn;
-  m_gu.w = (wm ? decode_weights_m(L, T) : gemm_pair_mode()) ? L->w13_128 : L->w13_256;
-  m_dn.w = (wm ? decode_weights_m(L, T) : gemm_pair_mode()) ? L->w2_128 : L->w2_256;
+  m_gu.w = (wm && decode_weights_m(L, T)) ? L->w13_128 : L->w13_256;
+  m_dn.w = (wm && decode_weights_m(L, T)) ? L->w2_128 : L->w2_256;
   memcpy(m_gu.t, W.tok_x, sizeof(m_gu.t));
   memcpy(m_dn.t, W.tok_act, sizeof(m_dn.t));
   const bool prof_saved = L->prof;
@@ -741,8 +781,8 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
   L->prof = false;  // stage marks describe moe_forward only
   EnumSource src = {nullptr, nullptr, 0, 0, 0};
   GemmMaps m_gu, m_dn;
-  m_gu.w = gemm_pair_mode() ? L->w13_128 : L->w13_256;
-  m_dn.w = gemm_pair_mode() ? L->w2_128 : L->w2_256;
+  m_gu.w = L->w13_256;
+  m_dn.w = L->w2_256;
 
   if (pruned_work) {
     const int rows_chunk = (int)align_up((size_t)K * Tc + (size_t)E * kTileRows, kTileRows);

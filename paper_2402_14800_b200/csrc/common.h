@@ -20,10 +20,7 @@ constexpr int kInterleave = 16;           // W1/W3 rows are interleaved in group
 constexpr int kDecodeMaxT = 256;          // up to here the small-batch path (weights read once) is used
 constexpr int kTokensDPerExpert = 40;      // small batches with this many tokens per expert or more: token-major decode GEMM
 constexpr int kTokensDMaxKept = 6;         // ... on layers with at most this many kept experts
-#ifndef MOE_DOWN_KB
-#define MOE_DOWN_KB 112
-#endif
-constexpr int kDecodeKbPerItem = MOE_DOWN_KB;  // k-blocks (of 64) per split-K item, decode down-proj
+constexpr int kDecodeKbPerItem = 112;      // k-blocks (of 64) per split-K item, decode down-proj
 
 // Device-resident description of one permuted batch, written by the scan kernel
 // (or by set_dense_meta for the search) and read by every later kernel.
@@ -47,7 +44,26 @@ struct KeptIds {
 // predecessor wrote (or still reads).  Every kernel on the forward path calls
 // pdl_launch_dependents() and pdl_wait() first thing (the GEMMs after their set-up), so the
 // stream order of all memory accesses is unchanged and only launch latency and prologues overlap.
+//
+// THE RULE for every kernel launched with launch_pdl: whatever an earlier kernel of the stream
+// may have written (token rows, routing records, permutation tables, the batch description,
+// activations, expert outputs, the residual) is read with ld_l2() below (ld.global.cg), never
+// through a `const T* __restrict__` parameter with a plain dereference or __ldg.  Such a kernel
+// is resident while its predecessors still write, no kernel boundary invalidates the SM's L1 in
+// between, and the non-coherent path (ld.global.nc, which the compiler may pick for const
+// __restrict__ data) is only defined for data that does not change during the kernel's lifetime:
+// an L1 line cached on this SM before the writer finished would be stale.  Only data that is
+// constant from the creation of the handle on (router rows, expert weights) keeps __ldg or the
+// streaming loads.  Operands that reach the SM through TMA are read at L2 by construction.
 #ifdef __CUDACC__
+__device__ __forceinline__ uint4 ld_l2(const uint4* p) { return __ldcg(p); }
+__device__ __forceinline__ float4 ld_l2(const float4* p) { return __ldcg(p); }
+__device__ __forceinline__ int ld_l2(const int32_t* p) { return __ldcg(p); }
+__device__ __forceinline__ float ld_l2(const float* p) { return __ldcg(p); }
+__device__ __forceinline__ int ld_l2(const uint8_t* p) { return (int)__ldcg(p); }
+__device__ __forceinline__ float ld_l2(const __nv_bfloat16* p) {
+  return __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p)) << 16);
+}
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -218,9 +234,9 @@ cudaError_t launch_simt_gate_up(const bf16* A, const bf16* W13, const GemmArgs& 
 cudaError_t launch_simt_down(const bf16* A, const bf16* W2, const GemmArgs& a, int cap_rows,
                              GemmOut out_kind, cudaStream_t st);
 cudaError_t gemm_set_attributes();
-// token-major GEMMs on CTA pairs (cta_group::2) instead of single CTAs
-void gemm_set_pair_mode(bool on);
-bool gemm_pair_mode();  // pair mode takes the weight maps with 128-row boxes (each CTA loads half a tile)
+// Test hook: one CTA runs the GEMMs' bounded wait on a barrier nobody arrives on, then their
+// abort path (see moe_test_hooks.h).
+cudaError_t launch_wait_expiry(int* status, unsigned long long limit_ns, cudaStream_t st);
 
 // ---- search (search.cu) ---------------------------------------------------------------
 // Where the enumeration finds the expert outputs.  Dense (topk_idx == null): Yall[T][E][h].

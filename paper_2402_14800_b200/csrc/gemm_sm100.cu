@@ -28,10 +28,7 @@ namespace {
 
 constexpr int BK = 64;            // k elements per pipeline stage = one 128-byte swizzle span
 constexpr int UMMA_K = 16;        // k elements per tcgen05.mma (bf16)
-#ifndef MOE_KBAND
-#define MOE_KBAND 16
-#endif
-constexpr int kBand = MOE_KBAND;  // row tiles that sweep the weight tiles together (L2 reuse)
+constexpr int kBand = 16;         // row tiles that sweep the weight tiles together (L2 reuse)
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;
 constexpr unsigned long long kDrainLimitNs = 2000000ull;
 
@@ -298,9 +295,6 @@ constexpr int TM_A_BYTES = 128 * 128;  // 128 token rows x 64 bf16
 constexpr int TM_B_BYTES = 256 * 128;  // 256 weight rows x 64 bf16
 constexpr int TM_STAGE = TM_A_BYTES + TM_B_BYTES;
 constexpr int TM_SMEM = TM_NS * TM_STAGE + 1024;
-#ifndef MOE_TM_KB_PAIRS
-#define MOE_TM_KB_PAIRS 1  // MMA issuer of the token-major kernel: two k-blocks per loop trip (0: one)
-#endif
 constexpr int TM_BN = 256;
 
 // Epilogue of one 128-row x 256-column accumulator tile of the token-major kernels: this
@@ -372,7 +366,7 @@ gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args)
   // everything above is independent of the preceding kernels; their results are read from here on
   pdl_wait();
   for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
-    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
+    reinterpret_cast<int32_t*>(&s_meta)[i] = ld_l2(reinterpret_cast<const int32_t*>(args.meta) + i);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -418,7 +412,6 @@ gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args)
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + buf * TM_BN;
       int kb = 0;
-#if MOE_TM_KB_PAIRS
       // two k-blocks per trip round the loop: both stages are awaited, then one fence, eight
       // MMAs, and the commit of each stage right after its own four
       for (; kb + 1 < KB; kb += 2, it += 2) {
@@ -445,7 +438,6 @@ gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args)
         __syncwarp();
       }
       if (!ok) break;
-#endif
       for (; kb < KB; ++kb, ++it) {
         const uint32_t s = it % TM_NS, ph = (it / TM_NS) & 1u;
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag));
@@ -490,285 +482,6 @@ gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args)
   teardown<TM_NS, 512>(bars, tmem_base, issued, args.status);
 }
 
-// ---------------------------------------------------------------------- gemm_tokens_m2
-//
-// The token-major GEMM on CTA pairs (cta_group::2): a cluster of two CTAs on neighbouring SMs
-// computes a 256-token x 256-weight-row tile.  Each CTA stages its own 128 token rows and its
-// own half (128 rows) of the weight tile, the leader CTA (cluster rank 0) issues one
-// M = 256 MMA that reads both CTAs' shared memory, and each CTA's tensor memory receives the
-// accumulator rows of its own tokens.  Per k-block a CTA loads 32 KB instead of the 48 KB of the
-// single-CTA tile, which is what limits that kernel at full clock.
-//   full[s]        in the leader; 1 arrival (leader's expect_tx of both CTAs' bytes) + tx bytes
-//   empty[s]       in each CTA; the leader's MMA commit arrives on both (commit to both CTAs)
-//   tmem_full[b]   in each CTA; the same
-//   tmem_empty[b]  in the leader; 8 arrivals (4 epilogue warps x 2 CTAs, the peer's remotely)
-// No TMA load carries more than one destination CTA.
-
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
-  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1,
-                                                 uint32_t bar_cluster) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster)
-      : "memory");
-}
-__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1,
-                                                 int c2, uint32_t bar_cluster) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3, %4}], [%5];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar_cluster)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst),
-               "r"(ncols)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish_pair() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
-               : "memory");
-}
-__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
-                                               uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n"
-      " .reg .pred p;\n"
-      " setp.ne.b32 p, %4, 0;\n"
-      " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
-      "}\n"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// arrives on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs
-// issued so far have completed
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-  const uint16_t both = 3;
-  asm volatile(
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-      ::"r"(bar), "h"(both)
-      : "memory");
-}
-
-constexpr int T2_NS = 6;
-constexpr int T2_A_BYTES = 128 * 128;  // this CTA's 128 token rows x 64 bf16
-constexpr int T2_B_BYTES = 128 * 128;  // this CTA's half of the 256 weight rows x 64 bf16
-constexpr int T2_STAGE = T2_A_BYTES + T2_B_BYTES;
-constexpr int T2_SMEM = T2_NS * T2_STAGE + 1024;
-constexpr int kBand2 = 8;  // pair tiles (256 rows) that sweep the weight tiles together
-
-struct TileM2 {
-  int c, nt, a_row, out_row, rows_valid;  // rows of the whole 256-row pair tile
-};
-
-// Pair tiles: every expert's 128-row tiles are taken two at a time.
-__device__ __forceinline__ int pair_tiles_total(const Meta& m, int r) {
-  int n = 0;
-  for (int c = 0; c < r; ++c) n += (m.tile_prefix[c + 1] - m.tile_prefix[c] + 1) >> 1;
-  return n;
-}
-__device__ __forceinline__ void decode_tile_m2(const Meta& m, const GemmArgs& a, int item, int Nt,
-                                               TileM2& t) {
-  int c = 0, before = 0;
-  for (;;) {
-    const int mt2 = (m.tile_prefix[c + 1] - m.tile_prefix[c] + 1) >> 1;
-    if (item < (before + mt2) * Nt || c + 1 >= a.r) break;
-    before += mt2;
-    ++c;
-  }
-  const int local = item - before * Nt;
-  const int Mt2 = (m.tile_prefix[c + 1] - m.tile_prefix[c] + 1) >> 1;
-  const int band = local / (kBand2 * Nt);
-  const int rem = local - band * kBand2 * Nt;
-  const int band_rows = min(kBand2, Mt2 - band * kBand2);
-  t.nt = rem / band_rows;
-  const int m2 = band * kBand2 + rem - t.nt * band_rows;
-  t.c = c;
-  t.a_row = a.a_row_base + a.a_off_mul * m.off[c] + 2 * kTileRows * m2;
-  t.out_row = a.out_row_base + a.out_off_mul * m.off[c] + 2 * kTileRows * m2;
-  t.rows_valid = min(2 * kTileRows, m.count[c] - 2 * kTileRows * m2);
-}
-
-template <bool GATE_UP, int OUT>
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_tokens_m2_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args) {
-  extern __shared__ uint8_t smem_raw[];
-  __shared__ Bars bars;
-  __shared__ Meta s_meta;
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();  // 0 = leader of the pair
-  const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < T2_NS; ++s) {
-      mbar_init(smem_u32(&bars.full[s]), 1);
-      mbar_init(smem_u32(&bars.empty[s]), 1);
-    }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&bars.tmem_full[i]), 1);
-      mbar_init(smem_u32(&bars.tmem_empty[i]), 8);
-    }
-    mbar_init(smem_u32(&bars.drain), 1);
-    bars.abort_flag = 0;
-    fence_barrier_init();
-    fence_proxy_async();
-  }
-  if (warp == 1) {
-    tmem_alloc_pair(smem_u32(&bars.tmem_base), 512);
-    tmem_relinquish_pair();
-  }
-  pdl_wait();
-  for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
-    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
-  tc_fence_before();
-  __syncthreads();
-  cluster_sync_all();  // both CTAs' barriers exist before anything is signalled across the pair
-  tc_fence_after();
-  const uint32_t tmem_base = *(volatile uint32_t*)&bars.tmem_base;
-  volatile int* abort_flag = &bars.abort_flag;
-  const uint32_t peer_abort = map_to_cta(smem_u32(&bars.abort_flag), rank ^ 1u);
-
-  const int KB = (args.K + BK - 1) / BK;
-  const int Nt = (args.n_w_rows + TM_BN - 1) / TM_BN;
-  const int n_items = pair_tiles_total(s_meta, args.r) * Nt;
-  uint32_t issued = 0;
-
-  if (warp == 0) {
-    // ---- TMA producer of this CTA's halves; completion is counted on the leader's barrier
-    uint32_t it = 0;
-    bool ok = true;
-    for (int item = cluster_id; item < n_items && ok; item += n_clusters) {
-      TileM2 t;
-      decode_tile_m2(s_meta, args, item, Nt, t);
-      for (int kb = 0; kb < KB; ++kb, ++it) {
-        const uint32_t s = it % T2_NS, ph = (it / T2_NS) & 1u;
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag));
-        if (!ok) break;
-        if (lane == 0) {
-          const uint32_t full_leader = map_to_cta(smem_u32(&bars.full[s]), 0);
-          const uint32_t sa = smem_base + s * T2_STAGE;
-          if (rank == 0) mbar_expect_tx(smem_u32(&bars.full[s]), 2 * T2_STAGE);
-          tma_load_2d_pair(sa, &maps.t[3], kb * BK, t.a_row + (int)rank * kTileRows, full_leader);
-          tma_load_3d_pair(sa + T2_A_BYTES, &maps.w, kb * BK, t.nt * TM_BN + (int)rank * 128, t.c,
-                           full_leader);
-        }
-        __syncwarp();
-      }
-    }
-    issued = it;
-  } else if (warp == 1) {
-    // ---- MMA issuer: only the leader; the peer's warp 1 owns that CTA's tensor memory
-    if (rank == 0) {
-      const uint32_t idesc = idesc_bf16(256, TM_BN);
-      uint32_t it = 0, tile_it = 0;
-      bool ok = true;
-      for (int item = cluster_id; item < n_items && ok; item += n_clusters, ++tile_it) {
-        const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_empty[buf]), bph ^ 1u, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * TM_BN;
-        for (int kb = 0; kb < KB; ++kb, ++it) {
-          const uint32_t s = it % T2_NS, ph = (it / T2_NS) & 1u;
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag));
-          if (!ok) break;
-          tc_fence_after();
-          if (lane == 0) {
-            const uint32_t sa = smem_base + s * T2_STAGE;
-            const uint64_t adesc = smem_desc_k128(sa);
-            const uint64_t bdesc = smem_desc_k128(sa + T2_A_BYTES);
-#pragma unroll
-            for (int k = 0; k < BK / UMMA_K; ++k)
-              umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-            umma_commit_pair(smem_u32(&bars.empty[s]));
-            if (kb == KB - 1) umma_commit_pair(smem_u32(&bars.tmem_full[buf]));
-          }
-          __syncwarp();
-        }
-      }
-    }
-  } else {
-    // ---- epilogue of this CTA's 128 token rows
-    const int wq = warp & 3;
-    const int row = 32 * wq + lane;
-    const uint32_t tmem_empty_leader0 = map_to_cta(smem_u32(&bars.tmem_empty[0]), 0);
-    const uint32_t tmem_empty_leader1 = map_to_cta(smem_u32(&bars.tmem_empty[1]), 0);
-    uint32_t tile_it = 0;
-    bool ok = true;
-    for (int item = cluster_id; item < n_items && ok; item += n_clusters, ++tile_it) {
-      TileM2 t;
-      decode_tile_m2(s_meta, args, item, Nt, t);
-      const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_full[buf]), bph, abort_flag));
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(32 * wq) << 16) + buf * TM_BN;
-      const int my_valid = min(kTileRows, max(0, t.rows_valid - (int)rank * kTileRows));
-      store_tile_tokens_m<GATE_UP, OUT>(taddr, args, t.nt, t.c, t.out_row + (int)rank * kTileRows,
-                                        my_valid, row);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(buf ? tmem_empty_leader1 : tmem_empty_leader0);
-    }
-  }
-
-  pdl_launch_dependents();
-  // ---- teardown: tell the partner if this CTA gave up, drain, and leave together (the leader's
-  // MMAs read the partner's shared memory and both tensor memories are freed as a pair)
-  tc_fence_before();
-  __syncthreads();
-  if (threadIdx.x == 0 && *(volatile int*)&bars.abort_flag) st_cluster_u32(peer_abort, 1u);
-  cluster_sync_all();
-  const int aborted = *(volatile int*)&bars.abort_flag;
-  if (aborted) {
-    if (warp == 0 && lane == 0 && rank == 0) {
-      int dummy = 0;
-      const uint32_t n = issued < (uint32_t)T2_NS ? issued : (uint32_t)T2_NS;
-      for (uint32_t i = 0; i < n; ++i) {
-        const uint32_t it = issued - 1 - i;
-        mbar_wait(smem_u32(&bars.full[it % T2_NS]), (it / T2_NS) & 1u, &dummy, kDrainLimitNs);
-      }
-    }
-    if (warp == 0 && lane == 0 && args.status) atomicExch(args.status, 1);
-    if (warp == 1 && lane == 0 && rank == 0) {
-      int dummy = 0;
-      umma_commit_pair(smem_u32(&bars.drain));
-      mbar_wait(smem_u32(&bars.drain), 0, &dummy, kDrainLimitNs);
-    }
-    __syncthreads();
-    cluster_sync_all();
-  }
-  if (warp == 1) {
-    tc_fence_after();
-    tmem_dealloc_pair(tmem_base, 512);
-  }
-}
-
 // ----------------------------------------------------------------------- gemm_weights_m
 
 // A pipeline stage holds two k-blocks (one barrier wait and one commit per 32 KB of weights: the
@@ -809,15 +522,9 @@ struct SchedW {
   int slot_floats;  // floats between the partial tiles of two slices
 };
 
-#ifndef MOE_SLICE_FIXED_KB
-#define MOE_SLICE_FIXED_KB 6
-#endif
-#ifndef MOE_FOLD_LOADS
-#define MOE_FOLD_LOADS 512
-#endif
 constexpr int kMinSliceKb = 4;                     // a slice covers at least this many k-blocks
-constexpr int kSliceFixedKb = MOE_SLICE_FIXED_KB;  // modelled fixed cost of a slice, in k-blocks
-constexpr int kFoldLoads = MOE_FOLD_LOADS;         // tokens x slices one thread adds up at most
+constexpr int kSliceFixedKb = 6;                   // modelled fixed cost of a slice, in k-blocks
+constexpr int kFoldLoads = 512;                    // tokens x slices one thread adds up at most
 constexpr int kTailHeaderFloats = (int)(kTailHeaderBytes / 4);  // arrival counters come first
 
 // Warp-collective: all 32 lanes of a converged warp call it and get the same result.
@@ -960,7 +667,7 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   // everything above is independent of the preceding kernels; their results are read from here on
   pdl_wait();
   for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
-    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
+    reinterpret_cast<int32_t*>(&s_meta)[i] = ld_l2(reinterpret_cast<const int32_t*>(args.meta) + i);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -974,9 +681,7 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
   if (warp == 0) {
     uint32_t it = 0;
     bool ok = true;
-#ifndef MOE_WM_NO_EVICT_FIRST
     const uint64_t evict_first = l2_policy_evict_first();
-#endif
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
       ItemW w;
       decode_item_w(s_meta, args, sched, item, w);
@@ -992,13 +697,9 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
           const uint32_t sa = smem_base + s * WM_STAGE;
           mbar_expect_tx(full, bytes * nk);
           for (int j = 0; j < nk; ++j) {
-#ifndef MOE_WM_NO_EVICT_FIRST
             // every weight byte is read exactly once: do not let it push the token rows, the
             // activations and the partial sums out of L2
             tma_load_3d_hint(sa + j * WM_A_BYTES, &maps.w, (kb + j) * BK, w.mt * 128, w.c, full, evict_first);
-#else
-            tma_load_3d(sa + j * WM_A_BYTES, &maps.w, (kb + j) * BK, w.mt * 128, w.c, full);
-#endif
             tma_load_2d(sa + 2 * WM_A_BYTES + j * WM_TOK_BYTES, &maps.t[w.bucket], (kb + j) * BK, w.tok_row, full);
           }
         }
@@ -1206,7 +907,7 @@ gemm_tokens_d_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args,
   }
   pdl_wait();
   for (int i = threadIdx.x; i < (int)(sizeof(Meta) / 4); i += blockDim.x)
-    reinterpret_cast<int32_t*>(&s_meta)[i] = reinterpret_cast<const int32_t*>(args.meta)[i];
+    reinterpret_cast<int32_t*>(&s_meta)[i] = ld_l2(reinterpret_cast<const int32_t*>(args.meta) + i);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -1371,6 +1072,39 @@ gemm_tokens_d_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args,
   teardown<TD_NS, 512>(bars, tmem_base, issued, args.status);
 }
 
+// ------------------------------------------------------------------ wait-expiry test hook
+
+// One CTA with the GEMMs' barrier block and a tensor-memory allocation.  Warp 0 waits, with the
+// GEMMs' own bounded wait, for phase 0 of a barrier on which nothing ever arrives; the wait runs
+// out after limit_ns, raises the abort flag, and the common teardown drains, reports and releases
+// tensor memory exactly as it does for a GEMM whose pipeline stalled.  Nothing is in flight, so
+// nothing can fault or spin beyond the limit.
+__global__ void __launch_bounds__(kThreads, 1)
+wait_expiry_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ Bars bars;
+  const int warp = threadIdx.x >> 5;
+  setup_barriers<1>(bars);
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars.tmem_base), 32);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *(volatile uint32_t*)&bars.tmem_base;
+  volatile int* abort_flag = &bars.abort_flag;
+  if (warp == 0) {
+    // the producer's wait of the GEMMs, on the phase that only an arrival could complete
+    (void)__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[0]), 0u, abort_flag, limit_ns));
+  } else if (warp == 1) {
+    // the other roles poll their own barriers and leave when the flag is up
+    (void)__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_empty[0]), 0u, abort_flag, 2 * limit_ns));
+  } else {
+    (void)__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_full[0]), 0u, abort_flag, 2 * limit_ns));
+  }
+  teardown<1, 32>(bars, tmem_base, 0u, status);
+}
+
 // ------------------------------------------------------------ CUDA-core debug kernels
 
 __device__ __forceinline__ float dot8(const uint4& a, const uint4& b, float acc) {
@@ -1429,10 +1163,9 @@ simt_down_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W2, GemmAr
 
 // ------------------------------------------------------------------------- tensor maps
 
-// L2 promotion size of every tensor map (a build-time knob for side-by-side measurements).
-#ifndef MOE_L2_PROMOTION
-#define MOE_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_256B
-#endif
+// Every tensor map asks for 256-byte L2 promotion (128 bytes or none measured 1.0-1.5 % slower
+// for the small-batch kernels and equal for the large-batch one).
+constexpr CUtensorMapL2promotion kL2Promotion = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -1462,7 +1195,7 @@ int make_map_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows,
   cuuint32_t es[2] = {1, 1};
   CUresult rc = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
                          strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         CU_TENSOR_MAP_SWIZZLE_128B, MOE_L2_PROMOTION,
+                         CU_TENSOR_MAP_SWIZZLE_128B, kL2Promotion,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? 0 : -(int)rc;
 }
@@ -1476,7 +1209,7 @@ int make_map_3d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows,
   cuuint32_t es[3] = {1, 1, 1};
   CUresult rc = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims,
                          strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         CU_TENSOR_MAP_SWIZZLE_128B, MOE_L2_PROMOTION,
+                         CU_TENSOR_MAP_SWIZZLE_128B, kL2Promotion,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? 0 : -(int)rc;
 }
@@ -1489,9 +1222,6 @@ cudaError_t gemm_set_attributes() {
   SET_ATTR((gemm_tokens_m_kernel<true, kOutActBf16>), TM_SMEM)
   SET_ATTR((gemm_tokens_m_kernel<false, kOutF32>), TM_SMEM)
   SET_ATTR((gemm_tokens_m_kernel<false, kOutBf16>), TM_SMEM)
-  SET_ATTR((gemm_tokens_m2_kernel<true, kOutActBf16>), T2_SMEM)
-  SET_ATTR((gemm_tokens_m2_kernel<false, kOutF32>), T2_SMEM)
-  SET_ATTR((gemm_tokens_m2_kernel<false, kOutBf16>), T2_SMEM)
   SET_ATTR((gemm_weights_m_kernel<true, 64>), WmCfg<64>::kSmem)
   SET_ATTR((gemm_weights_m_kernel<false, 64>), WmCfg<64>::kSmem)
   SET_ATTR((gemm_weights_m_kernel<true, 128>), WmCfg<128>::kSmem)
@@ -1505,38 +1235,14 @@ cudaError_t gemm_set_attributes() {
   return cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
 }
 
-// Launch on CTA pairs: cluster of 2, plain stream order.
-template <typename... KArgs, typename... Args>
-static cudaError_t launch_pair(void (*kernel)(KArgs...), int grid, size_t smem, cudaStream_t st,
-                               Args&&... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+cudaError_t launch_wait_expiry(int* status, unsigned long long limit_ns, cudaStream_t st) {
+  wait_expiry_kernel<<<1, kThreads, 0, st>>>(status, limit_ns);
+  return cudaGetLastError();
 }
-
-static bool g_pair_mode = false;
-void gemm_set_pair_mode(bool on) { g_pair_mode = on; }
-bool gemm_pair_mode() { return g_pair_mode; }
 
 cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps& maps,
                                  const GemmArgs& a, cudaStream_t st) {
   const int grid = g_num_sms > 0 ? g_num_sms : 148;
-  if (g_pair_mode) {
-    const int g2 = grid & ~1;
-    if (gate_up) return launch_pair(gemm_tokens_m2_kernel<true, kOutActBf16>, g2, T2_SMEM, st, maps, a);
-    if (out_kind == kOutF32) return launch_pair(gemm_tokens_m2_kernel<false, kOutF32>, g2, T2_SMEM, st, maps, a);
-    return launch_pair(gemm_tokens_m2_kernel<false, kOutBf16>, g2, T2_SMEM, st, maps, a);
-  }
   // Plain stream order for these long kernels: launched as programmatic dependents they measured
   // 3-5 % slower at T = 8192 (5.35 vs 5.0-5.1 ms per step), while the short kernels around them and
   // the weight-major kernels gain from the overlap.

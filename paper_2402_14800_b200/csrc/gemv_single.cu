@@ -34,17 +34,7 @@ __device__ __forceinline__ float dot8(const uint4& a, const uint4& w, float acc)
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 
 // Whatever an earlier kernel of the stream wrote (the token row, the activations, the routing
-// record, the residual) is read at L2 (ld.global.cg).  These kernels start as programmatic
-// dependents while their predecessor still runs, so their lifetime overlaps the writer's: the
-// non-coherent path (ld.global.nc) is only for data that never changes, and an L1 line cached
-// on this SM before the writer finished would be stale.
-__device__ __forceinline__ uint4 ld_l2(const uint4* p) { return __ldcg(p); }
-__device__ __forceinline__ int ld_l2(const int32_t* p) { return __ldcg(p); }
-__device__ __forceinline__ float ld_l2(const float* p) { return __ldcg(p); }
-__device__ __forceinline__ int ld_l2(const uint8_t* p) { return (int)__ldcg(p); }
-__device__ __forceinline__ float ld_l2(const bf16* p) {
-  return __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p)) << 16);
-}
+// record, the residual) is read with ld_l2 (see the rule beside launch_pdl).
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -7,10 +7,10 @@
 //   gather          copies the routed rows of x into expert-contiguous order.
 //   combine         Eq. 2: y = bf16(residual + w~_e0 o_e0 + w~_e1 o_e1), slot 0 first.
 //
-// The token rows (x) are read with ld.global.cg (L2), not through the non-coherent path: in a
-// stack the kernel that wrote them (RMSNorm, the previous layer's combine) may still be running
-// when these kernels start as its programmatic dependents, and an L1 line cached before the
-// writer finished would be stale.  The router rows never change and keep ld.global.nc.
+// Every kernel here that is launched as a programmatic dependent reads what earlier kernels of
+// the stream wrote with ld_l2 (the rule beside launch_pdl): token rows, routing records,
+// histograms, the batch description, expert outputs, the residual.  The router rows never
+// change and keep ld.global.nc.
 #include "common.h"
 #include "route_device.cuh"
 
@@ -22,7 +22,7 @@ namespace {
 // kernel costs a couple of memory round trips instead of a serial walk over the row.
 template <int R>
 __global__ void __launch_bounds__(256)
-router_small_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, int h, int r,
+router_small_kernel(const bf16* x, const bf16* __restrict__ Wg, int T, int h, int r,
                     float beta, KeptIds kept, RouteOut o) {
   pdl_launch_dependents();
   pdl_wait();
@@ -36,7 +36,7 @@ router_small_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
   const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)t * h);
   for (int v = threadIdx.x; v < nvec; v += 256) {
     float xf[8];
-    unpack8(__ldcg(xr + v), xf);
+    unpack8(ld_l2(xr + v), xf);
 #pragma unroll
     for (int c = 0; c < R; ++c) {
       if (c < r) {
@@ -74,7 +74,7 @@ router_small_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
 // records it writes are those of router_small_kernel + permute_gather_small_kernel for T = 1.
 template <int R>
 __global__ void __launch_bounds__(256)
-route_single_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int h, int r, float beta,
+route_single_kernel(const bf16* x, const bf16* __restrict__ Wg, int h, int r, float beta,
                     KeptIds kept, RouteOut o, int pad, Meta* meta, int32_t* __restrict__ pair_pos,
                     int32_t* __restrict__ row_token, bf16* __restrict__ xperm, int32_t* s_count,
                     int32_t* s_nskipped, int32_t* s_ntouched, int E) {
@@ -90,7 +90,7 @@ route_single_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
   const uint4* xr = reinterpret_cast<const uint4*>(x);
   for (int v = threadIdx.x; v < nvec; v += 256) {
     float xf[8];
-    unpack8(__ldcg(xr + v), xf);
+    unpack8(ld_l2(xr + v), xf);
 #pragma unroll
     for (int c = 0; c < R; ++c) {
       if (c < r) {
@@ -129,7 +129,7 @@ route_single_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
   uint4* d0 = reinterpret_cast<uint4*>(xperm + (size_t)p0 * h);
   uint4* d1 = reinterpret_cast<uint4*>(xperm + (size_t)(p1 < 0 ? p0 : p1) * h);
   for (int v = threadIdx.x; v < nvec; v += 256) {
-    const uint4 val = __ldcg(xr + v);
+    const uint4 val = ld_l2(xr + v);
     d0[v] = val;
     if (p1 >= 0) d1[v] = val;
   }
@@ -141,8 +141,7 @@ route_single_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int
 // Padding rows of the groups are left as they are: in the weight-major GEMM a token row only
 // feeds its own accumulator column, and the columns of padding rows are never stored.
 __global__ void __launch_bounds__(kDecodeMaxT)
-permute_gather_small_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ idx,
-                            const uint8_t* __restrict__ skipped, int T, int h, int r, int pad,
+permute_gather_small_kernel(const bf16* x, const int32_t* idx, const uint8_t* skipped, int T, int h, int r, int pad,
                             Meta* meta, int32_t* __restrict__ pair_pos,
                             int32_t* __restrict__ row_token, bf16* __restrict__ xperm,
                             int32_t* s_count, int32_t* s_nskipped, int32_t* s_ntouched, KeptIds kept,
@@ -159,8 +158,8 @@ permute_gather_small_kernel(const bf16* __restrict__ x, const int32_t* __restric
   {
     int e0 = -1, e1 = -1;
     if (i < T) {
-      e0 = idx[2 * i];
-      e1 = skipped[i] ? -1 : idx[2 * i + 1];
+      e0 = ld_l2(idx + 2 * i);
+      e1 = ld_l2(skipped + i) ? -1 : ld_l2(idx + 2 * i + 1);
     }
     s_e[i][0] = e0;
     s_e[i][1] = e1;
@@ -232,7 +231,7 @@ permute_gather_small_kernel(const bf16* __restrict__ x, const int32_t* __restric
   uint4* d0 = reinterpret_cast<uint4*>(xperm + (size_t)p0 * h);
   uint4* d1 = reinterpret_cast<uint4*>(xperm + (size_t)(p1 < 0 ? p0 : p1) * h);
   for (int v = i; v < nvec; v += blockDim.x) {
-    const uint4 val = __ldcg(src + v);
+    const uint4 val = ld_l2(src + v);
     d0[v] = val;
     if (p1 >= 0) d1[v] = val;
   }
@@ -245,7 +244,7 @@ permute_gather_small_kernel(const bf16* __restrict__ x, const int32_t* __restric
 
 template <int R>
 __global__ void __launch_bounds__(32 * kRouteTokPerBlock)
-router_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, int h, int r,
+router_kernel(const bf16* x, const bf16* __restrict__ Wg, int T, int h, int r,
               float beta, KeptIds kept, RouteOut o) {
   pdl_launch_dependents();
   pdl_wait();
@@ -265,7 +264,7 @@ router_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, in
     uint4 xv[kRouteXVec];
 #pragma unroll
     for (int i = 0; i < kRouteXVec; ++i)
-      xv[i] = (v0 + 32 * i < nvec) ? __ldcg(xr + v0 + 32 * i) : make_uint4(0u, 0u, 0u, 0u);
+      xv[i] = (v0 + 32 * i < nvec) ? ld_l2(xr + v0 + 32 * i) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
     for (int i = 0; i < kRouteXVec; ++i) {
       const int v = v0 + 32 * i;
@@ -324,7 +323,7 @@ router_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int T, in
 // gives every block its first position inside the expert's group; thread 0 then lays the
 // groups out (each padded to `pad` rows) and counts the 128-row tiles.
 __global__ void __launch_bounds__(1024)
-scan_kernel(const int32_t* __restrict__ blk_hist, int nblk, int r, int pad,
+scan_kernel(const int32_t* blk_hist, int nblk, int r, int pad,
             int32_t* __restrict__ blk_base, Meta* meta, int32_t* s_count, int32_t* s_nskipped,
             int32_t* s_ntouched, KeptIds kept, int E) {
   pdl_launch_dependents();
@@ -340,8 +339,8 @@ scan_kernel(const int32_t* __restrict__ blk_hist, int nblk, int r, int pad,
       const int b = b0 + lane;
       int v0 = 0, v1 = 0;
       if (b < nblk) {
-        v0 = blk_hist[(size_t)b * kHistCols + 2 * warp];
-        v1 = blk_hist[(size_t)b * kHistCols + 2 * warp + 1];
+        v0 = ld_l2(blk_hist + (size_t)b * kHistCols + 2 * warp);
+        v1 = ld_l2(blk_hist + (size_t)b * kHistCols + 2 * warp + 1);
       }
       const int v = v0 + v1;
       int inc = v;
@@ -360,7 +359,7 @@ scan_kernel(const int32_t* __restrict__ blk_hist, int nblk, int r, int pad,
     if (lane == 0) { s_tot[warp][0] = run0; s_tot[warp][1] = run - run0; }
   } else if (warp == kMaxE) {
     int n = 0;
-    for (int b = lane; b < nblk; b += 32) n += blk_hist[(size_t)b * kHistCols + 2 * kMaxE];
+    for (int b = lane; b < nblk; b += 32) n += ld_l2(blk_hist + (size_t)b * kHistCols + 2 * kMaxE);
 #pragma unroll
     for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(0xffffffffu, n, s);
     if (lane == 0) s_skipped = n;
@@ -403,8 +402,7 @@ scan_kernel(const int32_t* __restrict__ blk_hist, int nblk, int r, int pad,
 // Position of pair (t, slot) = start of its expert's group + pairs of that expert in earlier
 // blocks + pairs of that expert among the earlier tokens of this block.
 __global__ void __launch_bounds__(2 * kRouteTokPerBlock)
-scatter_kernel(const int32_t* __restrict__ idx, const uint8_t* __restrict__ skipped,
-               const int32_t* __restrict__ blk_base, const Meta* __restrict__ meta, int T,
+scatter_kernel(const int32_t* idx, const uint8_t* skipped, const int32_t* blk_base, const Meta* meta, int T,
                int32_t* __restrict__ pair_pos, int32_t* __restrict__ row_token) {
   pdl_launch_dependents();
   pdl_wait();
@@ -413,8 +411,8 @@ scatter_kernel(const int32_t* __restrict__ idx, const uint8_t* __restrict__ skip
   const int t = blockIdx.x * kRouteTokPerBlock + tl;
   int c = -1;
   if (t < T) {
-    c = idx[2 * t + slot];
-    if (slot == 1 && skipped[t]) c = -1;
+    c = ld_l2(idx + 2 * t + slot);
+    if (slot == 1 && ld_l2(skipped + t)) c = -1;
   }
   s_e[tl][slot] = c;
   __syncthreads();
@@ -423,7 +421,7 @@ scatter_kernel(const int32_t* __restrict__ idx, const uint8_t* __restrict__ skip
   if (c >= 0) {
     int rank = 0;
     for (int i = 0; i < tl; ++i) rank += (s_e[i][0] == c) + (s_e[i][1] == c);
-    pos = meta->off[c] + blk_base[(size_t)blockIdx.x * kMaxE + c] + rank;
+    pos = ld_l2(&meta->off[c]) + ld_l2(blk_base + (size_t)blockIdx.x * kMaxE + c) + rank;
     row_token[pos] = t;
   }
   pair_pos[2 * t + slot] = pos;
@@ -432,19 +430,19 @@ scatter_kernel(const int32_t* __restrict__ idx, const uint8_t* __restrict__ skip
 // -------------------------------------------------------------------------------- gather
 
 __global__ void __launch_bounds__(256)
-gather_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ row_token,
-              const Meta* __restrict__ meta, int h, bf16* __restrict__ xperm) {
+gather_kernel(const bf16* x, const int32_t* row_token, const Meta* meta, int h,
+              bf16* __restrict__ xperm) {
   pdl_launch_dependents();
   pdl_wait();
-  const int rows = meta->rows_total;
+  const int rows = ld_l2(&meta->rows_total);
   const int lane = threadIdx.x & 31;
   const int nvec = h >> 3;
   for (int row = blockIdx.x * 8 + (threadIdx.x >> 5); row < rows; row += gridDim.x * 8) {
-    const int t = row_token[row];
+    const int t = ld_l2(row_token + row);
     uint4* dst = reinterpret_cast<uint4*>(xperm + (size_t)row * h);
     if (t >= 0) {
       const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * h);
-      for (int v = lane; v < nvec; v += 32) dst[v] = __ldcg(src + v);
+      for (int v = lane; v < nvec; v += 32) dst[v] = ld_l2(src + v);
     } else {
       for (int v = lane; v < nvec; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
     }
@@ -454,14 +452,13 @@ gather_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ row_token,
 // ------------------------------------------------------------------------------- combine
 
 __global__ void __launch_bounds__(128)
-combine_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
-               const int32_t* __restrict__ pair_pos, const float* __restrict__ wn,
-               const bf16* residual, int T, int h, bf16* y) {
+combine_kernel(const float* O, int ksplit, size_t split_stride, const int32_t* pair_pos,
+               const float* wn, const bf16* residual, int T, int h, bf16* y) {
   pdl_launch_dependents();
   pdl_wait();
   const int t = blockIdx.x;
-  const int p0 = pair_pos[2 * t], p1 = pair_pos[2 * t + 1];
-  const float w0 = wn[2 * t], w1 = wn[2 * t + 1];
+  const int p0 = ld_l2(pair_pos + 2 * t), p1 = ld_l2(pair_pos + 2 * t + 1);
+  const float w0 = ld_l2(wn + 2 * t), w1 = ld_l2(wn + 2 * t + 1);
   const int nvec = h >> 3;
   for (int v = blockIdx.y * blockDim.x + threadIdx.x; v < nvec; v += gridDim.y * blockDim.x) {
     float a[8], b[8];
@@ -470,12 +467,12 @@ combine_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
 #pragma unroll 4
     for (int s = 0; s < ksplit; ++s) {
       const float4* o0 = reinterpret_cast<const float4*>(O + s * split_stride + (size_t)p0 * h) + 2 * v;
-      const float4 q0 = o0[0], q1 = o0[1];
+      const float4 q0 = ld_l2(o0), q1 = ld_l2(o0 + 1);
       a[0] += q0.x; a[1] += q0.y; a[2] += q0.z; a[3] += q0.w;
       a[4] += q1.x; a[5] += q1.y; a[6] += q1.z; a[7] += q1.w;
       if (p1 >= 0) {
         const float4* o1 = reinterpret_cast<const float4*>(O + s * split_stride + (size_t)p1 * h) + 2 * v;
-        const float4 r0 = o1[0], r1 = o1[1];
+        const float4 r0 = ld_l2(o1), r1 = ld_l2(o1 + 1);
         b[0] += r0.x; b[1] += r0.y; b[2] += r0.z; b[3] += r0.w;
         b[4] += r1.x; b[5] += r1.y; b[6] += r1.z; b[7] += r1.w;
       }
@@ -485,7 +482,7 @@ combine_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
     for (int k = 0; k < 8; ++k) z[k] = (p1 >= 0) ? fmaf(w1, b[k], w0 * a[k]) : w0 * a[k];
     if (residual) {
       float rf[8];
-      unpack8(reinterpret_cast<const uint4*>(residual + (size_t)t * h)[v], rf);
+      unpack8(ld_l2(reinterpret_cast<const uint4*>(residual + (size_t)t * h) + v), rf);
 #pragma unroll
       for (int k = 0; k < 8; ++k) z[k] += rf[k];
     }
@@ -519,7 +516,7 @@ router_topk_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int 
   const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)t * h);
   for (int v = threadIdx.x; v < nvec; v += 256) {
     float xf[8];
-    unpack8(__ldcg(xr + v), xf);
+    unpack8(ld_l2(xr + v), xf);
 #pragma unroll
     for (int c = 0; c < kMaxE; ++c) {
       if (c < r) {
@@ -679,20 +676,20 @@ coselection_kernel(const int32_t* __restrict__ idx, int T, int E, KeptIds kept,
 
 // D_t = || E_e0(x_t) - E_e1(x_t) ||_2, the quantity App. A.2 observes to be concentrated.
 __global__ void __launch_bounds__(256)
-top2_distance_kernel(const float* __restrict__ O, int ksplit, size_t split_stride,
-                     const int32_t* __restrict__ pair_pos, int T, int h, float* __restrict__ dist) {
+top2_distance_kernel(const float* O, int ksplit, size_t split_stride, const int32_t* pair_pos, int T,
+                     int h, float* __restrict__ dist) {
   __shared__ float s_part[8];
   pdl_launch_dependents();
   pdl_wait();
   const int t = blockIdx.x;
-  const int p0 = pair_pos[2 * t], p1 = pair_pos[2 * t + 1];
+  const int p0 = ld_l2(pair_pos + 2 * t), p1 = ld_l2(pair_pos + 2 * t + 1);
   float acc = 0.f;
   if (p1 >= 0) {
     for (int i = threadIdx.x; i < h; i += blockDim.x) {
       float a = 0.f, b = 0.f;
       for (int s = 0; s < ksplit; ++s) {
-        a += O[s * split_stride + (size_t)p0 * h + i];
-        b += O[s * split_stride + (size_t)p1 * h + i];
+        a += ld_l2(O + s * split_stride + (size_t)p0 * h + i);
+        b += ld_l2(O + s * split_stride + (size_t)p1 * h + i);
       }
       const float d = a - b;
       acc = fmaf(d, d, acc);
@@ -722,7 +719,7 @@ rmsnorm_kernel(const bf16* x, int T, int h, float eps, bf16* out) {
   float ss = 0.f;
   for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
     float f[8];
-    unpack8(xr[v], f);
+    unpack8(ld_l2(xr + v), f);
 #pragma unroll
     for (int k = 0; k < 8; ++k) ss = fmaf(f[k], f[k], ss);
   }
@@ -736,7 +733,7 @@ rmsnorm_kernel(const bf16* x, int T, int h, float eps, bf16* out) {
   const float inv = 1.0f / sqrtf(tot / (float)h + eps);
   for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
     float f[8];
-    unpack8(xr[v], f);
+    unpack8(ld_l2(xr + v), f);
     uint4 o;
     o.x = pack2(f[0] * inv, f[1] * inv); o.y = pack2(f[2] * inv, f[3] * inv);
     o.z = pack2(f[4] * inv, f[5] * inv); o.w = pack2(f[6] * inv, f[7] * inv);

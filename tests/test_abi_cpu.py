@@ -18,14 +18,18 @@ def lib():
 
 
 def declared_symbols():
-    src = open(os.path.join(ROOT, "include", "moe.h")).read()
-    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(moe_[a-z_0-9]+)\s*\(", src)))
+    import glob
+    names = set()
+    for path in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))):
+        src = re.sub(r"/\*.*?\*/", "", open(path).read(), flags=re.S)
+        names |= set(re.findall(r"\b(moe_[a-z_0-9]+)\s*\(", src))
+    return sorted(names)
 
 
 def test_every_declared_symbol_is_exported(lib):
     names = declared_symbols()
-    assert {"moe_layer_create", "moe_forward", "moe_prune_search"} <= set(names)
+    assert {"moe_layer_create", "moe_forward", "moe_prune_search", "moe_reserve",
+            "moe_test_wait_expiry", "moe_test_set_free_bytes_limit"} <= set(names)
     for n in names:
         assert hasattr(lib, n), n
 
@@ -67,6 +71,8 @@ def test_null_handle_is_an_error(lib):
     assert lib.moe_prune_search_multi(None, None, 4, None, 2, None, None) == -1
     assert lib.moe_calibrate_beta(None, None, 4, None) == -1
     assert lib.moe_device_status(None) == -1
+    assert lib.moe_reserve(None, 16) == -1
+    assert lib.moe_test_wait_expiry(None, 1000, 0) == -1
     assert lib.moe_layer_weight_bytes(None) == 0
     lib.moe_layer_destroy(None)
 

@@ -1,6 +1,6 @@
 """Alternative code paths behind switches, checked against the default path on the GPU:
-the CUDA-core debug kernels, the dense (all experts) search, the CTA-pair token-major GEMM,
-and replay of a captured CUDA graph of moe_forward."""
+the CUDA-core debug kernels, the dense (all experts) search, and replay of a captured CUDA
+graph of moe_forward."""
 import os
 
 import numpy as np
@@ -105,26 +105,6 @@ def test_dense_search_equals_pruned_work_search(weights, r):
     assert b0 == b1
 
 
-def test_cta_pair_gemm_agrees_with_single_cta_gemm(weights):
-    x = synth.make_tokens(1500, H, seed=5).to(DEV)
-    one = binding.MoeLayer(*weights)
-    y0 = one.forward(x, 0.3).clone()
-    l0, b0 = one.prune_search(x, 6)
-    one.close()
-    pair = layer_with_env(weights, MOE_GEMM_PAIR=1)
-    try:
-        y1 = pair.forward(x, 0.3)
-        l1, b1 = pair.prune_search(x, 6)
-        torch.cuda.synchronize()
-        assert pair.device_status() == 0
-    finally:
-        pair.close()
-        layer_with_env(weights, MOE_GEMM_PAIR=0).close()  # back to single CTAs for later tests
-    assert rel_l2(y1, y0) < 5e-3
-    np.testing.assert_allclose(l0, l1, rtol=1e-5)
-    assert b0 == b1
-
-
 @pytest.mark.parametrize("T", [1, 16, 600])
 def test_forward_replays_from_a_cuda_graph(weights, T):
     layer = binding.MoeLayer(*weights)
@@ -175,4 +155,131 @@ def test_back_to_back_calls_with_changing_inputs_equal_isolated_calls(weights, T
         for i in range(n):
             assert torch.equal(ys[i], want[i]), "step %d of round %d differs from the isolated call" % (i, rep)
     assert layer.device_status() == 0
+    layer.close()
+
+
+STACK_SPECS = [(20, 0xFF, 0.0), (21, 0b10111011, 0.4), (22, 0b00111100, 0.5)]
+
+
+@pytest.fixture(scope="module")
+def stack_layers():
+    build.build()
+    layers = []
+    for seed, kept, _ in STACK_SPECS:
+        W = synth.make_layer_weights(H, F, E, seed=seed)
+        layers.append(binding.MoeLayer(W.W_gate.to(DEV), W.W1.to(DEV), W.W3.to(DEV), W.W2.to(DEV), kept))
+    for l in layers[1:]:
+        l.share_scratch(layers[0])
+    yield layers
+    for l in reversed(layers):
+        l.close()
+
+
+@pytest.mark.parametrize("T", [1, 16, 128, 600])
+def test_queued_stack_steps_equal_isolated_calls(stack_layers, T):
+    # Three layers out of one set of scratch, every kernel a programmatic dependent of the one
+    # before, the state buffer read as the residual and overwritten by the same launch from the
+    # second layer on.  Steps are queued without synchronising, once on one refilled input buffer
+    # and once on separate inputs with no other kernel between two steps; each must reproduce the
+    # isolated call bit for bit.
+    n = 8
+    betas = [s[2] for s in STACK_SPECS]
+    xs = [synth.make_tokens(T, H, seed=400 + i).to(DEV) for i in range(n)]
+    want = []
+    for x in xs:
+        want.append(binding.stack_forward(stack_layers, x, betas, 1e-5).clone())
+        torch.cuda.synchronize()
+    x_buf = torch.empty_like(xs[0])
+    ys = [torch.empty_like(xs[0]) for _ in range(n)]
+    for rep in range(6 if T <= 128 else 3):
+        for i in range(n):
+            if rep % 2 == 0:
+                x_buf.copy_(xs[i])
+                binding.stack_forward(stack_layers, x_buf, betas, 1e-5, y=ys[i])
+            else:
+                binding.stack_forward(stack_layers, xs[i], betas, 1e-5, y=ys[i])
+        torch.cuda.synchronize()
+        for i in range(n):
+            assert torch.equal(ys[i], want[i]), "step %d of round %d differs from the isolated call" % (i, rep)
+        for y in ys:
+            y.zero_()
+    assert stack_layers[0].device_status() == 0
+
+
+@pytest.mark.parametrize("T", [1, 16, 128, 600])
+def test_queued_residual_steps_with_y_aliasing_the_residual(weights, T):
+    # state <- state + MoE(x) in place (y and residual are the same buffer), queued steps
+    n = 8
+    layer = binding.MoeLayer(*weights, 0b11110111)
+    xs = [synth.make_tokens(T, H, seed=500 + i).to(DEV) for i in range(n)]
+    s0 = synth.make_tokens(T, H, seed=599).to(DEV)
+    want, state = [], s0.clone()
+    for x in xs:
+        state = layer.forward(x, 0.4, residual=state).clone()   # separate output buffer, isolated
+        torch.cuda.synchronize()
+        want.append(state)
+    for rep in range(4):
+        state = s0.clone()
+        snaps = []
+        for i in range(n):
+            layer.forward(xs[i], 0.4, residual=state, y=state)
+            if rep % 2 == 0:
+                snaps.append(state.clone())
+        torch.cuda.synchronize()
+        assert torch.equal(state, want[-1]), "round %d" % rep
+        for i, snap in enumerate(snaps):
+            assert torch.equal(snap, want[i]), "step %d of round %d" % (i, rep)
+    assert layer.device_status() == 0
+    layer.close()
+
+
+@pytest.mark.parametrize("T", [2, 5, 16, 64, 128])
+def test_small_batches_repeat_many_queued_steps(weights, T):
+    # the small-batch sequences (router, permutation + gather, two GEMMs, combine: five programmatic
+    # dependents per step on the same scratch addresses) queued 200 steps deep on alternating inputs
+    layer = binding.MoeLayer(*weights, 0b11110111)
+    xa, xb = (synth.make_tokens(T, H, seed=s).to(DEV) for s in (610, 611))
+    wa, wb = layer.forward(xa, 0.4).clone(), layer.forward(xb, 0.4).clone()
+    torch.cuda.synchronize()
+    ya, yb = torch.empty_like(xa), torch.empty_like(xa)
+    bad = torch.zeros((), dtype=torch.int32, device=DEV)
+    for i in range(200):
+        if i % 2 == 0:
+            layer.forward(xa, 0.4, y=ya)
+            bad += (~torch.eq(ya, wa)).any().int()
+        else:
+            layer.forward(xb, 0.4, y=yb)
+            bad += (~torch.eq(yb, wb)).any().int()
+    torch.cuda.synchronize()
+    assert int(bad.item()) == 0
+    assert layer.device_status() == 0
+    layer.close()
+
+
+def test_reserve_makes_later_calls_allocation_free(weights):
+    # after moe_reserve(T_max) no forward call with T <= T_max grows the scratch, so a capture
+    # needs no warm-up call
+    layer = binding.MoeLayer(*weights)
+    layer.reserve(700)
+    held = layer.scratch_bytes
+    assert held > 0
+    s = torch.cuda.Stream(DEV)
+    layer.set_stream(s)
+    with torch.cuda.stream(s):
+        x = synth.make_tokens(700, H, seed=6).to(DEV)
+        y = torch.empty_like(x)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):       # first forward call of the handle, inside a capture
+            layer.forward(x, 0.4, y=y)
+        g.replay()
+        s.synchronize()
+        got = y.clone()
+        for T in (1, 2, 40, 256, 257, 700):
+            layer.forward(x[:T].contiguous(), 0.4)
+        s.synchronize()
+        assert layer.scratch_bytes == held
+        assert torch.equal(layer.forward(x, 0.4), got)
+        s.synchronize()
+    with pytest.raises(binding.MoeError):
+        layer.reserve(0)
     layer.close()
