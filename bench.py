@@ -6,7 +6,10 @@
 
 One step = one pass of the whole hot path (router, permutation, both grouped GEMMs, combine;
 or the pruning search) over one batch of seeded synthetic tokens at the Mixtral-8x7B layer
-shape.  Prints ONE JSON line.  With N > 1 (launched by torch.distributed.run) every rank runs
+shape.  Prints ONE JSON line.  The timed region is R blocks of exactly --steps steps (median
+block reported, best beside it).  The default run (decode, T = 128, all experts, beta = 0, one
+GPU) also measures the other configured workloads afterwards and reports them under "matrix":
+decode at other batch sizes and on pruned layers, prefill with skipping off and on, the search.  With N > 1 (launched by torch.distributed.run) every rank runs
 an independent replica on its own GPU: the path has no exchange step, so no collective sits
 on the data path; timing is the max over ranks.
 """
@@ -272,6 +275,303 @@ def run_reference(a):
 
 # -------------------------------------------------------------------------------- our arm
 
+def max_over_ranks_vec(v, dev=None):
+    """Element-wise max of a per-rank list over all ranks (identity for a single process)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(a) for a in v]
+    on_gpu = dist.get_backend() == "nccl"
+    t = torch.tensor(list(v), dtype=torch.float64, device=dev if on_gpu else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(a) for a in t.tolist()]
+
+
+def make_barrier(world, dev):
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+    return barrier
+
+
+def timed_blocks(step, steps, warmup, stream, dev, rank, local, world, target_s=1.5, max_s=20.0,
+                 min_repeats=30):
+    """W warm-up steps, then R blocks of exactly `steps` steps each, every block bracketed by a
+    barrier + device synchronisation on both sides and timed with CUDA events on the launching
+    stream (max over ranks per block).  R is chosen so that the blocks cover about `target_s`
+    seconds (at least `min_repeats`, fewer only when that would exceed `max_s`): a block of a few
+    milliseconds alone is a burst at full clock, the repeats reach the clock the board settles at
+    and give nvidia-smi time to sample it.  Returns the block times and the clock record."""
+    barrier = make_barrier(world, dev)
+    with torch.cuda.stream(stream):
+        for _ in range(max(warmup, 3)):
+            step()
+    barrier()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    with torch.cuda.stream(stream):
+        ev[0].record(stream)
+        for _ in range(steps):
+            step()
+        ev[1].record(stream)
+    barrier()
+    est_ms = max_over_ranks(ev[0].elapsed_time(ev[1]), dev)
+    R = max(min_repeats, int(np.ceil(target_s * 1e3 / max(est_ms, 1e-3))))
+    R = max(5, min(R, int(max_s * 1e3 / max(est_ms, 1e-3))))
+    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(R)]
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    for e0, e1 in events:
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(steps):
+                step()
+            e1.record(stream)
+        barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    blocks = max_over_ranks_vec([e0.elapsed_time(e1) for e0, e1 in events], dev)
+    return blocks, clocks
+
+
+def timing_record(blocks, steps, clocks):
+    med, best = float(np.median(blocks)), float(min(blocks))
+    rec = {"repeats": len(blocks), "steps_per_block": steps, "ms_per_step_median": med / steps,
+           "ms_per_step_best": best / steps, "ms_per_step_mean": float(np.mean(blocks)) / steps,
+           "how": "CUDA events around each block of `steps` steps, barrier + synchronise on both sides "
+                  "of every block, max over ranks per block; value and ms_per_step are the median block"}
+    if clocks and clocks.get("sm_mhz"):
+        # time x clock: comparable between a burst at full clock and a run at the power cap
+        rec["sm_cycles_per_step_median"] = med / steps * 1e-3 * clocks["sm_mhz"] * 1e6
+    return rec
+
+
+def decode_kernel_name(T, r_kept):
+    forced = os.environ.get("MOE_DECODE_KERNEL", "")
+    if T == 1 and single_token_gemv():
+        return "gemv_route_gate_up_kernel"
+    # the library's crossover: many tokens per expert -> token-major decode kernel
+    token_major = forced == "td" or (forced != "wm" and 2 * T >= 40 * r_kept and r_kept <= 6)
+    return "gemm_tokens_d_kernel<gate_up>" if token_major else "gemm_weights_m_kernel<gate_up>"
+
+
+def launches_per_forward(T):
+    # T = 1: routing + gate/up matrix-vector kernel, down kernel with the weighted sum
+    #   (with the GEMM path forced: routing, gate/up GEMM, down GEMM, combine);
+    # T <= 256: router, permute+gather, gate/up GEMM, down GEMM, combine;
+    # larger T: router, scan, scatter, gather, gate/up GEMM, down GEMM, combine
+    if T == 1:
+        return 2 if single_token_gemv() else 4
+    return 5 if T <= 256 else 7
+
+
+def forward_case(layer, x, y, beta, workload, wname, steps, warmup, stream, dev, rank, local, world, peaks,
+                 kept, target_s, max_s=20.0):
+    """One forward workload: routing facts, timed blocks, a pass with an event at every stage
+    boundary (per-kernel durations for the roofline), and the roofline record."""
+    from paper_2402_14800_b200 import binding
+    T = x.shape[0]
+    stats = binding.RoutingStats(T, E, dev)
+    with torch.cuda.stream(stream):
+        layer.forward(x, beta, y=y, stats=stats)
+    stream.synchronize()
+    pairs = 2 * T - int(stats.n_skipped.item())
+    touched = int(stats.n_experts_touched.item())
+
+    def step():
+        layer.forward(x, beta, y=y)
+
+    blocks, clocks = timed_blocks(step, steps, warmup, stream, dev, rank, local, world, target_s, max_s)
+    timing = timing_record(blocks, steps, clocks)
+    ms_step = timing["ms_per_step_median"]
+    # the same steps once more with an event at every stage boundary.  (The events sit between the
+    # kernels, so this pass does not overlap one kernel's launch with its predecessor's tail; the
+    # step time comes from the blocks above.)
+    n_prof = int(max(steps, min(2000, np.ceil(0.3e3 / max(ms_step, 1e-3)))))
+    layer.profile_enable(True)
+    with torch.cuda.stream(stream):
+        for _ in range(n_prof):
+            step()
+    stage_ms, ncalls = layer.profile_read()
+    layer.profile_enable(False)
+    if layer.device_status() != 0:
+        raise RuntimeError("a bounded wait inside a kernel expired during the timed steps")
+    gu_ms, dn_ms = stage_ms[1] / ncalls, stage_ms[2] / ncalls
+    stages = {"route_permute_ms": stage_ms[0] / ncalls, "gate_up_ms": gu_ms, "down_ms": dn_ms,
+              "combine_ms": stage_ms[3] / ncalls, "steps": ncalls}
+    r_kept = bin(kept).count("1")
+    if workload == "decode":
+        gu_bytes = touched * 2 * F * H * 2 + pairs * H * 2 + pairs * F * 2
+        dn_bytes = touched * H * F * 2 + pairs * F * 2 + 2 * pairs * H * 4
+        ach = gu_bytes / (gu_ms * 1e-3) / 1e9
+        kernel = decode_kernel_name(T, r_kept)
+        roofline = {"bound": "hbm", "kernel": kernel, "achieved": ach,
+                    "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"],
+                    "traffic": recorded_traffic(wname, kernel),
+                    "peak_source": peaks["source"], "algorithmic_bytes": gu_bytes,
+                    "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
+                    "down_kernel": {"achieved": dn_bytes / (dn_ms * 1e-3) / 1e9,
+                                    "frac": dn_bytes / (dn_ms * 1e-3) / 1e9 / peaks["hbm"]},
+                    "whole_step_frac": (gu_bytes + dn_bytes) / (ms_step * 1e-3) / 1e9 / peaks["hbm"]}
+    else:
+        gu_flop = pairs * 4 * H * F
+        dn_flop = pairs * 2 * H * F
+        ach = gu_flop / (gu_ms * 1e-3) / 1e12
+        step_tf = (gu_flop + dn_flop) / (ms_step * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel<gate_up>", "achieved": ach,
+                    "peak": peaks["tf_sust"], "unit": "TFLOP/s", "frac": ach / peaks["tf_sust"],
+                    "traffic": recorded_traffic(wname, "gemm_tokens_m_kernel<gate_up>"),
+                    "peak_source": peaks["source"] + " (sustained bf16; these runs sit at the power cap)",
+                    "frac_of_burst": ach / peaks["tf_burst"],
+                    "frac_of_nominal_dense_bf16": ach / NOMINAL_BF16_TFLOPS,
+                    "algorithmic_flop": gu_flop,
+                    "down_kernel": {"achieved": dn_flop / (dn_ms * 1e-3) / 1e12,
+                                    "frac": dn_flop / (dn_ms * 1e-3) / 1e12 / peaks["tf_sust"],
+                                    "frac_of_burst": dn_flop / (dn_ms * 1e-3) / 1e12 / peaks["tf_burst"]},
+                    "whole_step_tflops": step_tf,
+                    "whole_step_frac": step_tf / peaks["tf_sust"],
+                    "whole_step_frac_of_burst": step_tf / peaks["tf_burst"]}
+    return dict(T=T, beta=beta, pairs=pairs, touched=touched, timing=timing, clocks=clocks, stages=stages,
+                roofline=roofline, ms_step=ms_step, blocks=blocks)
+
+
+def search_case(layer, x, steps, warmup, stream, dev, rank, local, world, peaks, target_s, max_s=20.0):
+    """The pruning search for r = 6 and r = 4 over one evaluation of the experts."""
+    T = x.shape[0]
+
+    def step():
+        layer.prune_search_multi(x, [6, 4])
+
+    blocks, clocks = timed_blocks(step, steps, warmup, stream, dev, rank, local, world, target_s, max_s,
+                                  min_repeats=5)
+    timing = timing_record(blocks, steps, clocks)
+    ms_step = timing["ms_per_step_median"]
+    layer.profile_enable(True)
+    with torch.cuda.stream(stream):
+        for _ in range(max(2, min(steps, 5))):
+            step()
+    stage_ms, ncalls = layer.profile_read()
+    layer.profile_enable(False)
+    chunks = (T + 8191) // 8192
+    n_search = ncalls // (chunks + 1)   # a search records one set of marks per chunk and one for the enumerations
+    # r = 6 and r = 4 share one evaluation of each token's E - 4 + 2 = 6 top-ranked experts
+    dense = os.environ.get("MOE_SEARCH_DENSE", "") == "1"
+    K = E if dense else E - 4 + 2
+    gu_ms, dn_ms, en_ms = (stage_ms[i] / n_search for i in (1, 2, 3))
+    gu_flop, dn_flop = 4 * T * K * H * F, 2 * T * K * H * F
+    # the enumeration for r reads the E - r + 2 top-ranked expert outputs of every token once
+    en_bytes = T * H * 2 * ((E - 6 + 2) + (E - 4 + 2)) + 2 * T * E * 4
+    ach = gu_flop / (gu_ms * 1e-3) / 1e12
+    step_tf = (gu_flop + dn_flop) / (ms_step * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel<gate_up> (expert evaluations of the search)",
+                "achieved": ach, "peak": peaks["tf_sust"], "unit": "TFLOP/s", "frac": ach / peaks["tf_sust"],
+                "traffic": None, "frac_of_burst": ach / peaks["tf_burst"],
+                "frac_of_nominal_dense_bf16": ach / NOMINAL_BF16_TFLOPS,
+                "algorithmic_flop": gu_flop,
+                "peak_source": peaks["source"] + " (sustained bf16; these runs sit at the power cap)",
+                "down_kernel": {"achieved": dn_flop / (dn_ms * 1e-3) / 1e12,
+                                "frac": dn_flop / (dn_ms * 1e-3) / 1e12 / peaks["tf_sust"],
+                                "frac_of_burst": dn_flop / (dn_ms * 1e-3) / 1e12 / peaks["tf_burst"]},
+                "enumerate_kernel": {"bound": "hbm", "ms": en_ms, "algorithmic_bytes": en_bytes,
+                                     "achieved": en_bytes / (en_ms * 1e-3) / 1e9, "unit": "GB/s",
+                                     "frac": en_bytes / (en_ms * 1e-3) / 1e9 / peaks["hbm"]},
+                "whole_step_tflops": step_tf, "whole_step_frac": step_tf / peaks["tf_sust"],
+                "whole_step_frac_of_burst": step_tf / peaks["tf_burst"]}
+    stages = {"route_permute_ms": stage_ms[0] / n_search, "gate_up_ms": gu_ms, "down_ms": dn_ms,
+              "enumerate_ms": en_ms, "searches": n_search}
+    # per chunk: route, count, scan, scatter, gather, 2 GEMMs; then enumerate + reduce per size
+    return dict(T=T, timing=timing, clocks=clocks, stages=stages, roofline=roofline, ms_step=ms_step,
+                launches_per_step=chunks * 7 + 2 * 2)
+
+
+def matrix_rows(W, xcal, layers, stream, dev, rank, local, world, peaks, head):
+    """The other configured workloads, measured in the same invocation after the headline: decode
+    at T = 1 / 8 / 32 and on pruned layers, prefill at T = 2048 / 8192 / 32768 with skipping off
+    and on, the pruning search at T = 32768.  Each row has its own timed blocks, clock record and
+    roofline fractions; speed-ups are against the same kernels on the unpruned layer at beta = 0."""
+    from paper_2402_14800_b200 import binding
+    rows, base_ms = [], {}
+
+    def layer_for(kname):
+        if kname not in layers:
+            layers[kname] = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, KEPT[kname])
+            layers[kname].set_stream(stream)
+        return layers[kname]
+
+    betas = {}
+
+    def beta_for(kname, mode):
+        if mode == "0":
+            return 0.0
+        if kname not in betas:
+            betas[kname] = layer_for(kname).calibrate_beta(xcal)
+        return betas[kname]
+
+    plan = [("decode", 1, "full", "0"), ("decode", 1, "full", "calibrated"), ("decode", 8, "full", "0"),
+            ("decode", 32, "full", "0"), ("decode", 128, "full", "calibrated"), ("decode", 128, "r6", "0"),
+            ("decode", 128, "r4", "0"), ("decode", 128, "r4", "calibrated"),
+            ("prefill", 2048, "full", "0"), ("prefill", 2048, "full", "calibrated"),
+            ("prefill", 8192, "full", "0"), ("prefill", 8192, "full", "calibrated"),
+            ("prefill", 8192, "r4", "calibrated"),
+            ("prefill", 32768, "full", "0"), ("prefill", 32768, "full", "calibrated")]
+    base_ms[("decode", 128)] = head["ms_step"]
+    xs = {}
+    for workload, T, kname, mode in plan:
+        if T not in xs:
+            xs[T] = synth.make_tokens(T, H, seed=1, device=dev)
+        x = xs[T]
+        y = torch.empty_like(x)
+        steps = {"decode": 200, "prefill": max(3, 4096 * 10 // T)}[workload]
+        wname = "%s_T%d_%s_beta-%s" % (workload, T, kname, mode)
+        c = forward_case(layer_for(kname), x, y, beta_for(kname, mode), workload, wname, steps, 3, stream, dev,
+                         rank, local, world, peaks, KEPT[kname], target_s=1.2 if workload == "decode" else 2.0,
+                         max_s=6.0)
+        if kname == "full" and mode == "0":
+            base_ms[(workload, T)] = c["ms_step"]
+        rf = c["roofline"]
+        row = {"workload": wname, "tokens": T, "kept": kname, "beta": c["beta"], "pairs": c["pairs"],
+               "experts_touched": c["touched"], "tokens_per_s": T / (c["ms_step"] * 1e-3),
+               "ms_per_step": c["ms_step"], "ms_per_step_best": c["timing"]["ms_per_step_best"],
+               "repeats": c["timing"]["repeats"], "steps_per_block": steps,
+               "sm_cycles_per_step": c["timing"].get("sm_cycles_per_step_median"),
+               "bound": rf["bound"], "kernel": rf["kernel"], "unit": rf["unit"],
+               "gate_up_achieved": rf["achieved"], "gate_up_frac": rf["frac"],
+               "down_frac": rf["down_kernel"]["frac"], "whole_step_frac": rf["whole_step_frac"],
+               "stages": c["stages"], "clocks": c["clocks"]}
+        if rf["bound"] == "tensor":
+            row.update(flop_per_step=c["pairs"] * FLOP_PER_PAIR, whole_step_tflops=rf["whole_step_tflops"],
+                       gate_up_frac_of_burst=rf["frac_of_burst"],
+                       whole_step_frac_of_burst=rf["whole_step_frac_of_burst"],
+                       gate_up_frac_of_nominal_dense_bf16=rf["frac_of_nominal_dense_bf16"],
+                       peak_sustained=peaks["tf_sust"], peak_burst=peaks["tf_burst"])
+        else:
+            row.update(algorithmic_bytes=rf["algorithmic_bytes"], peak=peaks["hbm"])
+        b = base_ms.get((workload, T))
+        if b is not None and not (kname == "full" and mode == "0"):
+            row["speedup_vs_unpruned_beta0"] = b / c["ms_step"]
+        rows.append(row)
+        del y
+    xs.clear()
+    # the search (layer with all experts kept)
+    T = 32768
+    x = synth.make_tokens(T, H, seed=1, device=dev)
+    c = search_case(layer_for("full"), x, 3, 3, stream, dev, rank, local, world, peaks, target_s=1.5, max_s=8.0)
+    rf = c["roofline"]
+    rows.append({"workload": "search_T%d_r6+4" % T, "tokens": T, "subsets": 98,
+                 "subsets_tokens_per_s": 98 * T / (c["ms_step"] * 1e-3), "ms_per_step": c["ms_step"],
+                 "ms_per_step_best": c["timing"]["ms_per_step_best"], "repeats": c["timing"]["repeats"],
+                 "steps_per_block": 3, "sm_cycles_per_step": c["timing"].get("sm_cycles_per_step_median"),
+                 "bound": "tensor", "kernel": rf["kernel"], "unit": "TFLOP/s",
+                 "flop_per_step": 6 * T * 6 * H * F, "gate_up_achieved": rf["achieved"],
+                 "gate_up_frac": rf["frac"], "gate_up_frac_of_burst": rf["frac_of_burst"],
+                 "down_frac": rf["down_kernel"]["frac"], "whole_step_tflops": rf["whole_step_tflops"],
+                 "whole_step_frac": rf["whole_step_frac"], "whole_step_frac_of_burst": rf["whole_step_frac_of_burst"],
+                 "enumerate_kernel": rf["enumerate_kernel"], "peak_sustained": peaks["tf_sust"],
+                 "peak_burst": peaks["tf_burst"], "stages": c["stages"], "clocks": c["clocks"]})
+    return rows
+
+
 def run_ours(a):
     from paper_2402_14800_b200 import binding, build
     rank, world, local = dist_env()
@@ -284,6 +584,7 @@ def run_ours(a):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     peaks = measured_peaks()
+    barrier = make_barrier(world, dev)
 
     W, x, xcal = host_inputs(a, dev)
     kept = KEPT[a.kept]
@@ -295,70 +596,19 @@ def run_ours(a):
         beta = layer.calibrate_beta(xcal)
     T = a.tokens
     y = torch.empty_like(x)
-    stats = binding.RoutingStats(T, E, dev)
 
     if a.workload == "search":
-        def step():
-            # both subset sizes over one evaluation of the experts (moe_prune_search_multi)
-            layer.prune_search_multi(x, [6, 4])
-        launches_per_step = None
+        c = search_case(layer, x, a.steps, a.warmup, stream, dev, rank, local, world, peaks, a.target_seconds)
+        launches_per_step = c["launches_per_step"]
+        pairs = touched = 0
     else:
-        def step():
-            layer.forward(x, beta, y=y)
-        # T = 1: routing + gate/up matrix-vector kernel, down kernel with the weighted sum
-        #   (with the GEMM path forced: routing, gate/up GEMM, down GEMM, combine);
-        # T <= 256: router, permute+gather, gate/up GEMM, down GEMM, combine;
-        # larger T: router, scan, scatter, gather, gate/up GEMM, down GEMM, combine
-        single_gemv = a.tokens == 1 and single_token_gemv()
-        launches_per_step = (2 if single_gemv else 4) if a.tokens == 1 else (5 if a.tokens <= 256 else 7)
-
-    # routing facts for the algorithmic byte / flop counts (one untimed call)
-    pairs = touched = 0
-    if a.workload != "search":
-        layer.forward(x, beta, y=y, stats=stats)
-        stream.synchronize()
-        pairs = 2 * T - int(stats.n_skipped.item())
-        touched = int(stats.n_experts_touched.item())
-
-    def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
-        torch.cuda.synchronize(dev)
-
-    with torch.cuda.stream(stream):
-        for _ in range(max(a.warmup, 3)):
-            step()
-    barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    with torch.cuda.stream(stream):
-        ev0.record(stream)
-        for _ in range(a.steps):
-            step()
-        ev1.record(stream)
-    barrier()
-    ms_total = ev0.elapsed_time(ev1)
-    # the same K steps once more with an event at every stage boundary: per-kernel durations for
-    # the roofline.  (The events sit between the kernels, so this pass does not overlap one
-    # kernel's launch with its predecessor's tail; `value` comes from the pass above.)
-    stage_ms, ncalls = ([0, 0, 0, 0], 0)
-    if a.workload != "search":
-        layer.profile_enable(True)
-        with torch.cuda.stream(stream):
-            for _ in range(a.steps):
-                step()
-        stage_ms, ncalls = layer.profile_read()
-        layer.profile_enable(False)
-    if layer.device_status() != 0:
-        raise RuntimeError("a bounded wait inside a kernel expired during the timed steps")
-    clocks = sampler.stop() if rank == 0 else None
-    ms_total = max_over_ranks(ms_total, dev)
-    ms_step = ms_total / a.steps
-    value = whole_job_value(units_per_step(a), a.steps, ms_total, world)
+        c = forward_case(layer, x, y, beta, a.workload, workload_name(a), a.steps, a.warmup, stream, dev, rank,
+                         local, world, peaks, kept, a.target_seconds)
+        launches_per_step = launches_per_forward(T)
+        pairs, touched = c["pairs"], c["touched"]
+    ms_step = c["ms_step"]
+    value = whole_job_value(units_per_step(a), 1, ms_step, world)
+    timing, clocks, roofline, stages = c["timing"], c["clocks"], c["roofline"], c["stages"]
 
     # end to end through the host-buffer entry point (forward workloads only)
     e2e = None
@@ -367,73 +617,25 @@ def run_ours(a):
         yh = torch.empty_like(xh).pin_memory()
         for _ in range(3):
             layer.forward_host(xh, beta, yh)
-        barrier()
-        t0 = time.perf_counter()
         n_e2e = max(3, min(a.steps, 50))
-        for _ in range(n_e2e):
-            layer.forward_host(xh, beta, yh)
-        torch.cuda.synchronize(dev)
-        dt = time.perf_counter() - t0
-        dt = max_over_ranks(dt, dev)
+        reps = []
+        for _ in range(5):
+            barrier()
+            t0 = time.perf_counter()
+            for _ in range(n_e2e):
+                layer.forward_host(xh, beta, yh)
+            torch.cuda.synchronize(dev)
+            reps.append(time.perf_counter() - t0)
+        dt = float(np.median(max_over_ranks_vec(reps, dev)))
         e2e = {"value": world * T * n_e2e / dt, "unit": "tokens/s", "h2d_bytes_per_step": T * H * 2,
-               "d2h_bytes_per_step": T * H * 2, "timing": "host wall clock around the C-ABI call, max over ranks"}
+               "d2h_bytes_per_step": T * H * 2,
+               "timing": "host wall clock around %d C-ABI calls with host buffers, median of 5 such "
+                         "blocks, max over ranks" % n_e2e}
     else:
         # the search already returns its losses to host memory inside the timed call
         e2e = {"value": value, "unit": "subsets*tokens/s", "h2d_bytes_per_step": 0,
                "d2h_bytes_per_step": 98 * 4 + 8,
                "timing": "inputs resident on device; losses and argmin are copied to the host inside the call"}
-
-    # roofline of the dominant kernel (gate/up grouped GEMM), from the live per-stage events
-    roofline = None
-    stages = None
-    if a.workload != "search" and ncalls > 0:
-        gu_ms = stage_ms[1] / ncalls
-        dn_ms = stage_ms[2] / ncalls
-        stages = {"route_permute_ms": stage_ms[0] / ncalls, "gate_up_ms": gu_ms, "down_ms": dn_ms,
-                  "combine_ms": stage_ms[3] / ncalls}
-        if a.workload == "decode":
-            gu_bytes = touched * 2 * F * H * 2 + pairs * H * 2 + pairs * F * 2
-            dn_bytes = touched * H * F * 2 + pairs * F * 2 + 2 * pairs * H * 4
-            ach = gu_bytes / (gu_ms * 1e-3) / 1e9
-            forced = os.environ.get("MOE_DECODE_KERNEL", "")
-            r_kept = bin(KEPT[a.kept]).count("1")
-            # the library's crossover: many tokens per expert -> token-major decode kernel
-            token_major = forced == "td" or (forced != "wm" and 2 * a.tokens >= 40 * r_kept and r_kept <= 6)
-            kernel = "gemm_tokens_d_kernel<gate_up>" if token_major else "gemm_weights_m_kernel<gate_up>"
-            if single_gemv:  # one token: matrix-vector kernels on the CUDA cores
-                kernel = "gemv_route_gate_up_kernel"
-            roofline = {"bound": "hbm", "kernel": kernel, "achieved": ach,
-                        "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"],
-                        "traffic": recorded_traffic(workload_name(a), kernel),
-                        "peak_source": peaks["source"], "algorithmic_bytes": gu_bytes,
-                        "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
-                        "down_kernel": {"achieved": dn_bytes / (dn_ms * 1e-3) / 1e9,
-                                        "frac": dn_bytes / (dn_ms * 1e-3) / 1e9 / peaks["hbm"]},
-                        "whole_step_frac": (gu_bytes + dn_bytes) / (ms_step * 1e-3) / 1e9 / peaks["hbm"]}
-        else:
-            gu_flop = pairs * 4 * H * F
-            dn_flop = pairs * 2 * H * F
-            ach = gu_flop / (gu_ms * 1e-3) / 1e12
-            roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel<gate_up>", "achieved": ach,
-                        "peak": peaks["tf_sust"], "unit": "TFLOP/s", "frac": ach / peaks["tf_sust"],
-                        "traffic": recorded_traffic(workload_name(a), "gemm_tokens_m_kernel<gate_up>"),
-                        "peak_source": peaks["source"] + " (sustained bf16)",
-                        "frac_of_burst": ach / peaks["tf_burst"],
-                        "frac_of_nominal_dense_bf16": ach / NOMINAL_BF16_TFLOPS,
-                        "down_kernel": {"achieved": dn_flop / (dn_ms * 1e-3) / 1e12,
-                                        "frac": dn_flop / (dn_ms * 1e-3) / 1e12 / peaks["tf_sust"]},
-                        "whole_step_frac": (gu_flop + dn_flop) / (ms_step * 1e-3) / 1e12 / peaks["tf_sust"]}
-    elif a.workload == "search":
-        # r = 6 and r = 4 share one evaluation of each token's E - 4 + 2 = 6 top-ranked experts
-        dense = os.environ.get("MOE_SEARCH_DENSE", "") == "1"
-        flop = 6 * T * (E if dense else E - 4 + 2) * H * F
-        ach = flop / (ms_step * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel (expert evaluations of the search, whole step)",
-                    "achieved": ach, "peak": peaks["tf_sust"], "unit": "TFLOP/s",
-                    "frac": ach / peaks["tf_sust"], "traffic": None,
-                    "frac_of_burst": ach / peaks["tf_burst"],
-                    "frac_of_nominal_dense_bf16": ach / NOMINAL_BF16_TFLOPS,
-                    "peak_source": peaks["source"] + " (sustained bf16)"}
 
     # oracle on the host cores, bounded sample (rank 0, N = 1 only)
     cpu = None
@@ -447,6 +649,7 @@ def run_ours(a):
         per_unit = 98 if a.workload == "search" else 1
         cpu = {"value": n_sample * per_unit / dt, "unit": metric_unit(a)[1], "cores": O.num_threads(),
                "kind": "oracle", "sample": "%d of %d tokens, one pass, %.1f s" % (n_sample, T, dt)}
+        del Wh, xhb
 
     # reconstruction loss of the searched subset against the pruning baselines of the paper's
     # comparison (activation frequency, random), all on the same synthetic calibration batch
@@ -456,7 +659,7 @@ def run_ours(a):
         counts = layer.coselection(x)
         baselines = {}
         for r_, (losses, best) in zip((6, 4), layer.prune_search_multi(x, [6, 4])):
-            masks = [sum(1 << i for i in c) for c in combinations(range(E), r_)]
+            masks = [sum(1 << i for i in c_) for c_ in combinations(range(E), r_)]
             fmask = layer.frequency_subset(counts, r_)
             baselines["r%d" % r_] = {"searched_subset": best, "searched_loss": min(losses),
                                      "frequency_subset": fmask, "frequency_loss": losses[masks.index(fmask)],
@@ -468,13 +671,19 @@ def run_ours(a):
         baselines["top2_distance"] = {"tokens": int(d.numel()), "mean": float(d.mean()),
                                       "std_over_mean": float(d.std() / d.mean())}
 
+    # the rest of the configured workloads (single GPU, default workload only)
+    matrix = None
+    if a.matrix and world == 1 and rank == 0 and workload_name(a) == "decode_T128_full_beta-0":
+        layers = {a.kept: layer}
+        t0 = time.perf_counter()
+        matrix = matrix_rows(W, xcal, layers, stream, dev, rank, local, world, peaks, c)
+        for k, l in layers.items():
+            if l is not layer:
+                l.close()
+        matrix_s = time.perf_counter() - t0
+
     if rank == 0:
         metric, unit = metric_unit(a)
-        gpu_launches = launches_per_step * a.steps if launches_per_step else None
-        if a.workload == "search":
-            chunks = (T + 8191) // 8192
-            # per chunk: route, count, scan, scatter, gather, 2 GEMMs; then enumerate + reduce per size
-            gpu_launches = a.steps * (chunks * 7 + 2 * 2)
         line = {
             "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": a.steps,
             "warmup": max(a.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
@@ -485,11 +694,16 @@ def run_ours(a):
                        "l2": "per step the kernels stream %.2f GB of weights, far above the 126 MB L2"
                              % (touched * 3 * H * F * 2 / 1e9) if a.workload != "search" else
                              "inputs and intermediates are GBs, far above the 126 MB L2"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "roofline": roofline,
+            "timing": timing, "clocks": clocks, "e2e": e2e,
+            "gpu_launches": launches_per_step * a.steps * timing["repeats"],
+            "gpu_launches_per_step": launches_per_step, "roofline": roofline,
             "cpu_baseline": cpu, "stages": stages,
         }
         if baselines:
             line["pruning_baselines"] = baselines
+        if matrix is not None:
+            line["matrix"] = matrix
+            line["matrix_wall_s"] = matrix_s
         print(json.dumps(line), flush=True)
     layer.close()
     if world > 1:
@@ -694,6 +908,10 @@ def main():
     ap.add_argument("--search-r", default="6+4")
     ap.add_argument("--ref-sample", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-matrix", dest="matrix", action="store_false",
+                    help="headline workload only (the default decode run also measures the other configured workloads)")
+    ap.add_argument("--target-seconds", type=float, default=1.5,
+                    help="device time the repeated blocks of the timed region should cover")
     a = ap.parse_args()
     if a.tokens is None:
         a.tokens = {"decode": 128, "prefill": 8192, "search": 32768, "stack": 16}[a.workload]

@@ -281,6 +281,10 @@ int moe_stack_forward(moe_layer_t* const* layers, int n_layers, const void* x, i
  *   stage 1  gate/up grouped GEMM with the SwiGLU epilogue
  *   stage 2  down-projection grouped GEMM
  *   stage 3  combine (Eq. 2)
+ * The searches record too: per chunk of 8192 calibration tokens one set of marks
+ * (stage 0 routing + permutation, 1 gate/up GEMM, 2 down GEMM, 3 empty) and one
+ * more set for the enumerations (stages 0-2 empty, 3 enumeration + reduction),
+ * so a search of n chunks counts as n + 1 calls.
  * moe_profile_read synchronises the stream, writes the milliseconds summed over
  * the calls recorded since the last enable/read into stage_ms[MOE_PROFILE_STAGES]
  * and their number into *calls (host memory), and starts a new window.  At most

@@ -777,8 +777,10 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
   if ((rc = grow(L, W.s_losses, (size_t)nC * 4))) return rc;
   if ((rc = grow(L, W.s_meta, sizeof(Meta)))) return rc;
   Meta* meta = (Meta*)W.s_meta.p;
+  // While profiling, every chunk records one set of stage marks (permutation, gate/up, down, an
+  // empty fourth stage) and the enumerations one more (three empty stages, then stage 3).
   const bool prof_saved = L->prof;
-  L->prof = false;  // stage marks describe moe_forward only
+  if (L->prof && (L->prof_used % (MOE_PROFILE_STAGES + 1)) != 0) L->prof_used = 0;
   EnumSource src = {nullptr, nullptr, 0, 0, 0};
   GemmMaps m_gu, m_dn;
   m_gu.w = L->w13_256;
@@ -804,6 +806,7 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
       int32_t* idx = (int32_t*)W.k_idx.p + (size_t)t0 * K;
       int32_t* nact = (int32_t*)W.k_nact.p + t0;
       int32_t* pos = (int32_t*)W.k_pos.p + (size_t)t0 * K;
+      mark(L);
       // beta = -1: the skipping rule never fires, every token keeps its K top-ranked experts
       cudaError_t e = launch_router_topk(xc, L->Wg, rows, h, E, K, -1.0f, L->kept, idx,
                                          (float*)W.k_wn.p + (size_t)t0 * K, nact, nullptr, nullptr,
@@ -822,6 +825,7 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
         L->prof = prof_saved;
         return fail(MOE_ERR_CUDA, "search permutation: %s", cudaGetErrorString(e));
       }
+      mark(L);
       GemmArgs gu, dn;
       memset(&gu, 0, sizeof(gu));
       memset(&dn, 0, sizeof(dn));
@@ -833,6 +837,8 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
         L->prof = prof_saved;
         return rc;
       }
+      mark(L);
+      mark(L);
     }
     src.topk_idx = (const int32_t*)W.k_idx.p;
     src.pair_pos = (const int32_t*)W.k_pos.p;
@@ -859,10 +865,13 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
     memset(&ro, 0, sizeof(ro));
     ro.idx = (int32_t*)W.idx.p; ro.wn = (float*)W.wn.p; ro.ratio = (float*)W.ratio.p;
     ro.skipped = (uint8_t*)W.skipped.p; ro.logits = (float*)W.s_logits.p;
+    mark(L);
     CUDA_TRY(launch_router((const bf16*)x_calib, L->Wg, T, h, E, 0.f, L->kept, ro, st));
     for (int t0 = 0; t0 < T; t0 += Tc) {
       const int rows = (T - t0) < Tc ? (T - t0) : Tc;
+      if (t0 > 0) mark(L);
       CUDA_TRY(launch_set_dense_meta(meta, E, rows, Tc_pad, st));
+      mark(L);
       GemmArgs gu, dn;
       memset(&gu, 0, sizeof(gu));
       memset(&dn, 0, sizeof(dn));
@@ -874,9 +883,12 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
         L->prof = prof_saved;
         return rc;
       }
+      mark(L);
+      mark(L);
     }
   }
   L->prof = prof_saved;
+  for (int i = 0; i < MOE_PROFILE_STAGES; ++i) mark(L);
   // one enumeration per subset size over the same expert outputs
   std::vector<std::vector<uint32_t>> masks(n_r);
   size_t o = 0;
@@ -890,6 +902,7 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
     CUDA_TRY(cudaMemcpyAsync(losses + o, L->ws->s_losses.p, n * 4, cudaMemcpyDeviceToHost, st));
     o += n;
   }
+  mark(L);
   if ((rc = check_status(L))) return rc;
   o = 0;
   for (int i = 0; i < n_r; ++i) {
