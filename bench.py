@@ -111,18 +111,22 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             pass
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             try:
                 sm.append(float(r[0])); mx.append(float(r[1]))
             except Exception:
                 continue
+            try:
+                pw.append(float(r[2]))
+            except Exception:
+                pass
             for n, v in zip(names, r[4:8]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
-                    samples=len(sm), reasons=sorted(reasons))
+                    samples=len(sm), power_w=float(np.median(pw)) if pw else None, reasons=sorted(reasons))
 
 
 def dist_env():
@@ -295,8 +299,11 @@ def make_barrier(world, dev):
     return barrier
 
 
+MIN_REPEATS = 30  # blocks of the timed region at least (--min-repeats)
+
+
 def timed_blocks(step, steps, warmup, stream, dev, rank, local, world, target_s=1.5, max_s=20.0,
-                 min_repeats=30):
+                 min_repeats=None):
     """W warm-up steps, then R blocks of exactly `steps` steps each, every block bracketed by a
     barrier + device synchronisation on both sides and timed with CUDA events on the launching
     stream (max over ranks per block).  R is chosen so that the blocks cover about `target_s`
@@ -316,8 +323,10 @@ def timed_blocks(step, steps, warmup, stream, dev, rank, local, world, target_s=
         ev[1].record(stream)
     barrier()
     est_ms = max_over_ranks(ev[0].elapsed_time(ev[1]), dev)
+    if min_repeats is None:
+        min_repeats = MIN_REPEATS
     R = max(min_repeats, int(np.ceil(target_s * 1e3 / max(est_ms, 1e-3))))
-    R = max(5, min(R, int(max_s * 1e3 / max(est_ms, 1e-3))))
+    R = max(min(5, min_repeats), min(R, int(max_s * 1e3 / max(est_ms, 1e-3))))
     events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(R)]
     sampler = ClockSampler(local)
     if rank == 0:
@@ -388,7 +397,7 @@ def forward_case(layer, x, y, beta, workload, wname, steps, warmup, stream, dev,
     # the same steps once more with an event at every stage boundary.  (The events sit between the
     # kernels, so this pass does not overlap one kernel's launch with its predecessor's tail; the
     # step time comes from the blocks above.)
-    n_prof = int(max(steps, min(2000, np.ceil(0.3e3 / max(ms_step, 1e-3)))))
+    n_prof = int(max(steps, min(2000, np.ceil(min(0.3, target_s) * 1e3 / max(ms_step, 1e-3)))))
     layer.profile_enable(True)
     with torch.cuda.stream(stream):
         for _ in range(n_prof):
@@ -444,7 +453,7 @@ def search_case(layer, x, steps, warmup, stream, dev, rank, local, world, peaks,
         layer.prune_search_multi(x, [6, 4])
 
     blocks, clocks = timed_blocks(step, steps, warmup, stream, dev, rank, local, world, target_s, max_s,
-                                  min_repeats=5)
+                                  min_repeats=min(5, MIN_REPEATS))
     timing = timing_record(blocks, steps, clocks)
     ms_step = timing["ms_per_step_median"]
     layer.profile_enable(True)
@@ -734,8 +743,29 @@ def run_stack(a):
     x = synth.make_tokens(T, H, seed=1, device=dev)
     state = synth.make_tokens(a.cal_tokens, H, seed=1001, device=dev)
     layers, betas, masks, search_ms = [], [], [], 0.0
-    state_p = state.clone() if (r < 8 and a.search_mode == "progressive") else None
-    for l in range(NL):
+    # the result of an earlier search of the same stack (masks, losses, betas) is reloaded
+    # instead of searching again: the pruned layers are then built straight from the masks
+    from paper_2402_14800_b200 import pruning_io
+    pmeta = {"E": E, "r": r, "n_layers": NL, "h": H, "f": F, "calibration_tokens": a.cal_tokens,
+             "search_mode": a.search_mode if r < 8 else "none", "beta": a.beta, "weight_seed0": 100,
+             "calibration_seed": 1001}
+    pfile = a.pruning_file or "pruning_stack%d_%s_%s_%s_cal%d.json" % (NL, a.kept, a.search_mode, a.beta, a.cal_tokens)
+    loaded = None
+    if r < 8 and os.path.exists(pfile) and not a.research:
+        loaded = pruning_io.load_pruning(pfile, expect_meta=pmeta)
+    all_losses = []
+    state_p = state.clone() if (r < 8 and a.search_mode == "progressive" and loaded is None) else None
+    if loaded is not None:
+        for l in range(NL):
+            W = synth.make_layer_weights(H, F, E, seed=100 + l, device=dev)
+            layer = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, loaded[l]["kept_mask"])
+            if layers:
+                layer.share_scratch(layers[0])
+            layers.append(layer)
+            masks.append(loaded[l]["kept_mask"])
+            betas.append(loaded[l]["beta"])
+            del W
+    for l in range(NL if loaded is None else 0):
         W = synth.make_layer_weights(H, F, E, seed=100 + l, device=dev)
         xn = binding.rmsnorm(state)
         xn_cal = xn
@@ -753,13 +783,14 @@ def run_stack(a):
             t0 = time.perf_counter()
             if state_p is None:
                 # layer-wise: every layer is searched on the unpruned stack's states
-                _, mask = full.prune_search(xn, r)
+                losses_l, mask = full.prune_search(xn, r)
             else:
                 # progressive: input from the pruned stack so far, target from the unpruned stack
                 F_ref = full.forward(xn, 0.0).float()
                 xn_cal = binding.rmsnorm(state_p)
-                _, mask = full.prune_search_progressive(xn_cal, F_ref, r)
+                losses_l, mask = full.prune_search_progressive(xn_cal, F_ref, r)
                 del F_ref
+            all_losses.append(losses_l)
             search_ms += 1e3 * (time.perf_counter() - t0)
             state = full.forward(xn, 0.0, residual=state)
             torch.cuda.synchronize(dev)
@@ -773,9 +804,14 @@ def run_stack(a):
         masks.append(mask)
         layers.append(layer)
         del W
+    if r < 8 and loaded is None and rank == 0:
+        pruning_io.save_pruning(pfile, pmeta, [{"kept_mask": m, "losses": ls, "beta": b}
+                                               for m, ls, b in zip(masks, all_losses, betas)])
     # how far the pruned stack's calibration states ended up from the unpruned stack's
     drift = None
-    if state_p is not None:
+    if loaded is not None:
+        pass
+    elif state_p is not None:
         drift = float((state_p.float() - state.float()).norm() / state.float().norm())
     elif r < 8:
         sp = synth.make_tokens(a.cal_tokens, H, seed=1001, device=dev)
@@ -783,7 +819,7 @@ def run_stack(a):
             sp = layer.forward(binding.rmsnorm(sp), 0.0, residual=sp)
         drift = float((sp.float() - state.float()).norm() / state.float().norm())
         del sp
-    del state, xn
+    del state
     stream = torch.cuda.Stream(dev)
     for layer in layers:
         layer.set_stream(stream)
@@ -876,6 +912,8 @@ def run_stack(a):
                        "betas": [round(b, 4) for b in betas], "weight_bytes": weight_bytes,
                        "experts_touched_sum": sum(touched), "pairs_sum": sum(pairs),
                        "search_ms_total": search_ms, "calibration_tokens": a.cal_tokens,
+                       "pruning_file": (pfile if r < 8 else None),
+                       "pruning_reloaded": loaded is not None,
                        "search_mode": a.search_mode if r < 8 else None,
                        "final_state_rel_error_vs_unpruned": drift,
                        "parallelism": "replicas x%d, no collective" % world,
@@ -902,6 +940,10 @@ def main():
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--cal-tokens", type=int, default=4096)
     ap.add_argument("--search-mode", default="layerwise", choices=["layerwise", "progressive"])
+    ap.add_argument("--pruning-file", default=None,
+                    help="stack workload: JSON with the per-layer kept masks, losses and betas; reloaded when it "
+                         "exists and matches, written after a search (default: a name derived from the configuration)")
+    ap.add_argument("--research", action="store_true", help="stack workload: search again even if the file exists")
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--beta", default="0", choices=["0", "calibrated"])
     ap.add_argument("--kept", default="full", choices=list(KEPT))
@@ -910,9 +952,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-matrix", dest="matrix", action="store_false",
                     help="headline workload only (the default decode run also measures the other configured workloads)")
+    ap.add_argument("--min-repeats", type=int, default=30,
+                    help="blocks of --steps steps in the timed region at least (1 with --target-seconds 0 for a profiler)")
     ap.add_argument("--target-seconds", type=float, default=1.5,
                     help="device time the repeated blocks of the timed region should cover")
     a = ap.parse_args()
+    global MIN_REPEATS
+    MIN_REPEATS = max(1, a.min_repeats)
     if a.tokens is None:
         a.tokens = {"decode": 128, "prefill": 8192, "search": 32768, "stack": 16}[a.workload]
     if a.steps is None:

@@ -262,8 +262,10 @@ int check_status(moe_layer* L) {
 // The two grouped GEMMs of the experts over a batch described by `meta`.
 int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmMaps& m_gu,
                      const GemmMaps& m_dn, GemmArgs gu, GemmArgs dn, GemmOut dn_kind,
-                     const bf16* gu_A, const bf16* dn_A, int simt_rows, int T = 0) {
+                     const bf16* gu_A, const bf16* dn_A, int simt_rows, int T = 0, int est_rows = 0) {
   gu.meta = meta; dn.meta = meta;
+  // rows of the batch at most (by default the capacity in rows, which bounds the pairs that run)
+  gu.est_rows = dn.est_rows = est_rows > 0 ? est_rows : simt_rows;
   gu.r = L->r; dn.r = L->r;
   gu.K = L->h; gu.n_w_rows = 2 * L->f;
   dn.K = L->f; dn.n_w_rows = L->h;
@@ -745,11 +747,11 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
     return fail(MOE_ERR_INVALID_ARG, "the search needs a layer created with all %d experts kept", L->E);
   if (!rs || n_r < 1 || n_r > kMaxE) return fail(MOE_ERR_INVALID_ARG, "no subset sizes given (or more than %d)", kMaxE);
   int r = L->E;  // the smallest size: it needs the most experts evaluated per token
-  long nC = 0;   // the largest number of subsets of any size
+  long nC = 0;   // subsets of all sizes together
   for (int i = 0; i < n_r; ++i) {
     if (rs[i] < 2 || rs[i] > L->E) return fail(MOE_ERR_INVALID_ARG, "r = %d outside 2..%d", rs[i], L->E);
     if (rs[i] < r) r = rs[i];
-    if (binom(L->E, rs[i]) > nC) nC = binom(L->E, rs[i]);
+    nC += binom(L->E, rs[i]);
   }
   const int E = L->E, h = L->h, f = L->f;
   cudaStream_t st = L->stream;
@@ -759,12 +761,8 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
   const int Tc = T < 8192 ? T : 8192;  // tokens per chunk of expert evaluations
   const int Tc_pad = (int)align_up((size_t)Tc, kTileRows);
   const int nchunks = (T + Tc - 1) / Tc;
-  size_t partial_floats = 0;  // per-block partial losses of the largest enumeration
-  for (int i = 0; i < n_r; ++i) {
-    const size_t n = (size_t)binom(E, rs[i]);
-    const size_t need = (size_t)enumerate_num_blocks(T, (int)n) * n;
-    if (need > partial_floats) partial_floats = need;
-  }
+  // per-block partial losses of the enumeration
+  const size_t partial_floats = (size_t)enumerate_num_blocks(T, (int)nC) * (size_t)nC;
   // A subset of r experts always contains two of a token's K = E - r + 2 top-ranked experts,
   // so only those K need to be evaluated per token (all of them when K = E).
   const int K = E - r + 2;
@@ -879,7 +877,7 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
       dn.a_off_mul = 1; dn.out_row_base = t0; dn.out_off_mul = 0; dn.out_col_mul = h;
       dn.out_ld = (long long)E * h; dn.out = W.s_yall.p;
       if ((rc = run_expert_gemms(L, meta, false, m_gu, m_dn, gu, dn, kOutBf16, xa,
-                                 (const bf16*)W.s_act.p, rows))) {
+                                 (const bf16*)W.s_act.p, rows, 0, E * rows))) {
         L->prof = prof_saved;
         return rc;
       }
@@ -889,19 +887,24 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
   }
   L->prof = prof_saved;
   for (int i = 0; i < MOE_PROFILE_STAGES; ++i) mark(L);
-  // one enumeration per subset size over the same expert outputs
+  // One enumeration for all subset sizes over the same expert outputs.  Which pair of experts a
+  // subset routes a token to depends on the subset alone (its two highest-ranked kept experts,
+  // which lie within the token's E - r + 2 <= K top-ranked ones), so the subsets of every size go
+  // through one pass that reads each token's K expert outputs once; every loss is computed by
+  // the same operations in the same order as in a pass of its own size.
   std::vector<std::vector<uint32_t>> masks(n_r);
-  size_t o = 0;
+  std::vector<uint32_t> all_masks;
   for (int i = 0; i < n_r; ++i) {
     masks[i] = subset_masks(E, rs[i]);
-    const size_t n = masks[i].size();
-    CUDA_TRY(cudaMemcpyAsync(W.s_subsets.p, masks[i].data(), n * 4, cudaMemcpyHostToDevice, st));
-    CUDA_TRY(launch_enumerate((const float*)W.s_logits.p, (const bf16*)W.s_yall.p, T, E, rs[i], h,
-                              (const uint32_t*)W.s_subsets.p, (int)n, (float*)W.s_partial.p,
-                              (double*)W.s_loss_sq.p, (float*)W.s_losses.p, F_ref, src, st));
-    CUDA_TRY(cudaMemcpyAsync(losses + o, L->ws->s_losses.p, n * 4, cudaMemcpyDeviceToHost, st));
-    o += n;
+    all_masks.insert(all_masks.end(), masks[i].begin(), masks[i].end());
   }
+  const size_t n_all = all_masks.size();
+  CUDA_TRY(cudaMemcpyAsync(W.s_subsets.p, all_masks.data(), n_all * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(launch_enumerate((const float*)W.s_logits.p, (const bf16*)W.s_yall.p, T, E, r, h,
+                            (const uint32_t*)W.s_subsets.p, (int)n_all, (float*)W.s_partial.p,
+                            (double*)W.s_loss_sq.p, (float*)W.s_losses.p, F_ref, src, st));
+  CUDA_TRY(cudaMemcpyAsync(losses, L->ws->s_losses.p, n_all * 4, cudaMemcpyDeviceToHost, st));
+  size_t o = 0;
   mark(L);
   if ((rc = check_status(L))) return rc;
   o = 0;

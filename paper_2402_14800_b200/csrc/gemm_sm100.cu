@@ -217,7 +217,7 @@ struct Bars {
 };
 
 template <int NS>
-__device__ __forceinline__ void setup_barriers(Bars& b) {
+__device__ __forceinline__ void setup_barriers(Bars& b, uint32_t tmem_empty_arrivals = 4) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(smem_u32(&b.full[s]), 1);
@@ -225,7 +225,7 @@ __device__ __forceinline__ void setup_barriers(Bars& b) {
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&b.tmem_full[i]), 1);
-      mbar_init(smem_u32(&b.tmem_empty[i]), 4);
+      mbar_init(smem_u32(&b.tmem_empty[i]), tmem_empty_arrivals);
     }
     mbar_init(smem_u32(&b.drain), 1);
     b.abort_flag = 0;
@@ -236,8 +236,8 @@ __device__ __forceinline__ void setup_barriers(Bars& b) {
 
 // Common tail: after an abort, wait (bounded) for loads and MMAs that are still in flight,
 // report, and release tensor memory.
-template <int NS, int TMEM_COLS>
-__device__ __forceinline__ void teardown(Bars& b, uint32_t tmem_base, uint32_t issued,
+template <int TMEM_COLS>
+__device__ __forceinline__ void teardown(Bars& b, uint32_t tmem_base, uint32_t issued, uint32_t NS,
                                          int* status) {
   tc_fence_before();
   __syncthreads();
@@ -247,7 +247,7 @@ __device__ __forceinline__ void teardown(Bars& b, uint32_t tmem_base, uint32_t i
     if (warp == 0 && lane == 0) {
       // the last min(issued, NS) stages may still have a load in flight
       int dummy = 0;
-      const uint32_t n = issued < (uint32_t)NS ? issued : (uint32_t)NS;
+      const uint32_t n = issued < NS ? issued : NS;
       for (uint32_t i = 0; i < n; ++i) {
         const uint32_t it = issued - 1 - i;
         mbar_wait(smem_u32(&b.full[it % NS]), (it / NS) & 1u, &dummy, kDrainLimitNs);
@@ -268,89 +268,129 @@ __device__ __forceinline__ void teardown(Bars& b, uint32_t tmem_base, uint32_t i
 }
 
 // ------------------------------------------------------------------------ gemm_tokens_m
+//
+// Large batches.  One CTA computes 256 token rows x 256 weight rows per item: per k-block of 64
+// it stages two 128-row token tiles and one 256-row weight tile (64 KB) and issues eight MMAs,
+// four into each of two accumulators that together fill all 512 tensor-memory columns.  What
+// bounds this kernel is the traffic from L2 to shared memory and its latency (measured: with 2 /
+// 3 / 4 stages of a 128 x 256 tile the tensor pipe was busy in proportion to the stages, and an
+// L2 prefetch stream made it slower), so the tile is as large as tensor memory allows: a
+// 256 x 256 tile moves 2/3 of the bytes of a 128 x 256 tile per FLOP, and three stages of it
+// cover 3 x 1024 pipe cycles of latency instead of 4 x 512.  The price is that the accumulators
+// are not double-buffered: the MMAs of the next item wait until the epilogue warps have read the
+// previous item out of tensor memory, which is why there are many epilogue warps (each reads
+// 32 lanes x 128 or 64 columns) and why accumulator 0 is released before accumulator 1.
+// An item whose second 128 rows are all padding (an expert group's odd last row tile) runs as
+// a half item: no second token tile, no MMAs into accumulator 1.
 
 struct TileM {
-  int c, nt, a_row, out_row, rows_valid;
+  int c, nt, a_row, out_row, rows_valid;  // rows_valid in 1 .. 256
 };
 
-__device__ __forceinline__ void decode_tile_m(const Meta& m, const GemmArgs& a, int item, int Nt,
-                                              TileM& t) {
-  int c = 0;
-  while (c + 1 < a.r && m.tile_prefix[c + 1] * Nt <= item) ++c;
-  const int local = item - m.tile_prefix[c] * Nt;
-  const int Mt = m.tile_prefix[c + 1] - m.tile_prefix[c];
-  const int band = local / (kBand * Nt);
-  const int rem = local - band * kBand * Nt;
-  const int band_rows = min(kBand, Mt - band * kBand);
-  t.nt = rem / band_rows;
-  const int mt = band * kBand + rem - t.nt * band_rows;
-  t.c = c;
-  t.a_row = a.a_row_base + a.a_off_mul * m.off[c] + kTileRows * mt;
-  t.out_row = a.out_row_base + a.out_off_mul * m.off[c] + kTileRows * mt;
-  t.rows_valid = min(kTileRows, m.count[c] - kTileRows * mt);
-}
-
-constexpr int TM_NS = 4;
-constexpr int TM_A_BYTES = 128 * 128;  // 128 token rows x 64 bf16
-constexpr int TM_B_BYTES = 256 * 128;  // 256 weight rows x 64 bf16
+constexpr int TM_NS = 3;
+constexpr int TM_A_HALF = 128 * 128;        // 128 token rows x 64 bf16
+constexpr int TM_A_BYTES = 2 * TM_A_HALF;   // two token tiles
+constexpr int TM_B_BYTES = 256 * 128;       // 256 weight rows x 64 bf16
 constexpr int TM_STAGE = TM_A_BYTES + TM_B_BYTES;
 constexpr int TM_SMEM = TM_NS * TM_STAGE + 1024;
 constexpr int TM_BN = 256;
+// Epilogue warps per CTA: 2 accumulators x 4 tensor-memory lane quarters x 1 or 2 column halves.
+// The SwiGLU epilogue (an exponential and a division per output) is the long one and, with the
+// accumulators single-buffered, sits on the critical path between two items: 16 warps (gate/up
+// launch 11.3 vs 12.2 ms at 32768 tokens).  The plain copies of the down projection were
+// 4 % faster with 8 (5.48 vs 5.72 ms): its items are 3.5 times as long, and fewer warps wait.
+template <bool GATE_UP> struct TmCfg {
+  static constexpr int kEpiWarps = GATE_UP ? 16 : 8;
+  static constexpr int kThreads = 64 + 32 * kEpiWarps;
+};
 
-// Epilogue of one 128-row x 256-column accumulator tile of the token-major kernels: this
-// thread owns tensor-memory lane `row` (one token row) and walks the 256 columns in chunks of 32.
+// An item covers `unit` row tiles of 128 (2 normally; 1 for launches with too few items to fill
+// the machine with double row tiles, see launch_gemm_tokens_m).  Items of expert c:
+// ceil(row tiles / unit) x Nt weight tiles, ordered band of kBand / unit row items -> weight
+// tile -> row item, so that the items in flight share few token tiles and weight tiles in L2.
+__device__ __forceinline__ void decode_tile_m(const Meta& m, const GemmArgs& a, int item, int Nt,
+                                              int unit, TileM& t) {
+  int c = 0, first = 0;
+  for (;;) {
+    const int mtu = (m.tile_prefix[c + 1] - m.tile_prefix[c] + unit - 1) / unit;
+    if (c + 1 >= a.r || item < first + mtu * Nt) break;
+    first += mtu * Nt;
+    ++c;
+  }
+  const int local = item - first;
+  const int Mtu = (m.tile_prefix[c + 1] - m.tile_prefix[c] + unit - 1) / unit;
+  const int band_items = kBand / unit;
+  const int band = local / (band_items * Nt);
+  const int rem = local - band * band_items * Nt;
+  const int band_rows = min(band_items, Mtu - band * band_items);
+  t.nt = rem / band_rows;
+  const int mt = band * band_items + rem - t.nt * band_rows;
+  const int rows = unit * kTileRows;
+  t.c = c;
+  t.a_row = a.a_row_base + a.a_off_mul * m.off[c] + rows * mt;
+  t.out_row = a.out_row_base + a.out_off_mul * m.off[c] + rows * mt;
+  t.rows_valid = min(rows, m.count[c] - rows * mt);
+}
+
+__device__ __forceinline__ int num_items_m(const Meta& m, const GemmArgs& a, int Nt, int unit) {
+  int n = 0;
+  for (int c = 0; c < a.r; ++c) n += ((m.tile_prefix[c + 1] - m.tile_prefix[c] + unit - 1) / unit) * Nt;
+  return n;
+}
+
+// Epilogue of 128 accumulator rows x columns [32 j0, 32 j1) of one accumulator: this thread owns
+// tensor-memory lane `row` (one token row) and walks the columns in chunks of 32.
 template <bool GATE_UP, int OUT>
 __device__ __forceinline__ void store_tile_tokens_m(uint32_t taddr, const GemmArgs& args, int nt, int c,
-                                                    int out_row, int rows_valid, int row) {
+                                                    int out_row, int rows_valid, int row, int j0, int j1) {
   const bool row_ok = row < rows_valid;
   const long long orow = (long long)(out_row + row) * args.out_ld + (long long)c * args.out_col_mul;
 #pragma unroll 1
-      for (int j = 0; j < TM_BN / 32; ++j) {
-        const int col0 = nt * TM_BN + 32 * j;  // first weight row of this chunk
-        if (col0 >= args.n_w_rows) break;        // warp-uniform
-        uint32_t v[32];
-        tmem_ld32(taddr + 32 * j, v);
-        tmem_ld_wait();
-        if (GATE_UP) {
-          // chunk = 16 gate rows then 16 up rows of the features col0/2 .. col0/2 + 15
-          uint32_t o[8];
+  for (int j = j0; j < j1; ++j) {
+    const int col0 = nt * TM_BN + 32 * j;  // first weight row of this chunk
+    if (col0 >= args.n_w_rows) break;        // warp-uniform
+    uint32_t v[32];
+    tmem_ld32(taddr + 32 * j, v);
+    tmem_ld_wait();
+    if (GATE_UP) {
+      // chunk = 16 gate rows then 16 up rows of the features col0/2 .. col0/2 + 15
+      uint32_t o[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const float a0 = silu_mul(__uint_as_float(v[2 * i]), __uint_as_float(v[16 + 2 * i]));
-            const float a1 = silu_mul(__uint_as_float(v[2 * i + 1]), __uint_as_float(v[17 + 2 * i]));
-            o[i] = pack_bf16(a0, a1);
-          }
-          if (row_ok) {
-            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(args.out) + orow + (col0 >> 1));
-            dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-            dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-          }
-        } else if (OUT == kOutF32) {
-          if (row_ok) {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.out) + orow + col0);
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-              dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                   __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
-          }
-        } else {
-          if (row_ok) {
-            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(args.out) + orow + col0);
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              dst[i] = make_uint4(
-                  pack_bf16(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
-                  pack_bf16(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
-                  pack_bf16(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
-                  pack_bf16(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
-          }
-        }
+      for (int i = 0; i < 8; ++i) {
+        const float a0 = silu_mul(__uint_as_float(v[2 * i]), __uint_as_float(v[16 + 2 * i]));
+        const float a1 = silu_mul(__uint_as_float(v[2 * i + 1]), __uint_as_float(v[17 + 2 * i]));
+        o[i] = pack_bf16(a0, a1);
       }
+      if (row_ok) {
+        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(args.out) + orow + (col0 >> 1));
+        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+      }
+    } else if (OUT == kOutF32) {
+      if (row_ok) {
+        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.out) + orow + col0);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                               __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+      }
+    } else {
+      if (row_ok) {
+        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(args.out) + orow + col0);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          dst[i] = make_uint4(
+              pack_bf16(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
+              pack_bf16(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
+              pack_bf16(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
+              pack_bf16(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
+      }
+    }
+  }
 }
 
-
 template <bool GATE_UP, int OUT>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(TmCfg<GATE_UP>::kThreads, 1)
 gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ Bars bars;
@@ -358,7 +398,9 @@ gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args)
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  setup_barriers<TM_NS>(bars);
+  // tmem_empty[a]: one arrival per epilogue warp of accumulator a
+  constexpr int TM_EPI_WARPS = TmCfg<GATE_UP>::kEpiWarps;
+  setup_barriers<4>(bars, TM_EPI_WARPS / 2);
   if (warp == 1) {
     tmem_alloc(smem_u32(&bars.tmem_base), 512);
     tmem_relinquish();
@@ -375,111 +417,142 @@ gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args)
 
   const int KB = (args.K + BK - 1) / BK;
   const int Nt = (args.n_w_rows + TM_BN - 1) / TM_BN;
-  const int n_items = s_meta.tile_prefix[args.r] * Nt;
+  // single row tiles per item: 4 stages of 48 KB (one token tile + the weight tile), every item
+  // a half item; the accumulators then alternate, which double-buffers them
+  const bool single = args.single_row_tiles != 0;
+  const int unit = single ? 1 : 2;
+  const uint32_t ns = single ? 4u : (uint32_t)TM_NS;
+  const uint32_t stage_bytes = single ? (uint32_t)(TM_A_HALF + TM_B_BYTES) : (uint32_t)TM_STAGE;
+  const uint32_t b_off = single ? (uint32_t)TM_A_HALF : (uint32_t)TM_A_BYTES;
+  const int n_items = num_items_m(s_meta, args, Nt, unit);
   uint32_t issued = 0;
 
   if (warp == 0) {
     // ---- TMA producer
-    uint32_t it = 0;
+    uint32_t it = 0, s = 0, ph = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
       TileM t;
-      decode_tile_m(s_meta, args, item, Nt, t);
+      decode_tile_m(s_meta, args, item, Nt, unit, t);
+      const bool full_item = t.rows_valid > kTileRows;
+      const uint32_t bytes = TM_B_BYTES + (full_item ? TM_A_BYTES : TM_A_HALF);
       for (int kb = 0; kb < KB; ++kb, ++it) {
-        const uint32_t s = it % TM_NS, ph = (it / TM_NS) & 1u;
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag));
         if (!ok) break;
         if (lane == 0) {
           const uint32_t full = smem_u32(&bars.full[s]);
-          const uint32_t sa = smem_base + s * TM_STAGE;
-          mbar_expect_tx(full, TM_STAGE);
+          const uint32_t sa = smem_base + s * stage_bytes;
+          mbar_expect_tx(full, bytes);
           tma_load_2d(sa, &maps.t[3], kb * BK, t.a_row, full);
-          tma_load_3d(sa + TM_A_BYTES, &maps.w, kb * BK, t.nt * TM_BN, t.c, full);
+          tma_load_3d(sa + b_off, &maps.w, kb * BK, t.nt * TM_BN, t.c, full);
+          if (full_item) tma_load_2d(sa + TM_A_HALF, &maps.t[3], kb * BK, t.a_row + kTileRows, full);
         }
+        if (++s == ns) { s = 0; ph ^= 1u; }
         __syncwarp();
       }
     }
     issued = it;
   } else if (warp == 1) {
-    // ---- MMA issuer
+    // ---- MMA issuer.  A full item uses both accumulators (rows 0-127 in accumulator 0, rows
+    // 128-255 in accumulator 1); half items take the accumulators in turn.  n0 / n1 count the
+    // uses of each accumulator, nh the half items; the epilogue warps count the same way.
+    // The loop of this warp, not the tensor pipe, sets the pace whenever it spends more than about
+    // one MMA's time between two MMAs (the pipe queues little beyond the MMA it executes), so the
+    // body of a k-block is kept short, and the commit that releases a stage is issued after the
+    // first MMA of the NEXT k-block instead of between two k-blocks, where it would sit next to
+    // the wait for the next stage's data.  A commit covers every MMA issued before it, so the
+    // stage is released slightly later than it could be, never earlier.  (Measured side by side:
+    // the deferred commit 5 % faster; the loop run by one lane with the others parked, or the wait
+    // for the next stage moved between the MMAs as well, each 4-7 % slower.)
     const uint32_t idesc = idesc_bf16(128, TM_BN);
-    uint32_t it = 0, tile_it = 0;
+    uint32_t s = 0, ph = 0, n0 = 0, n1 = 0, nh = 0;
+    uint32_t owed_bar = 0;  // empty barrier of the stage whose release is still to be committed
     bool ok = true;
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile_it) {
-      const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_empty[buf]), bph ^ 1u, abort_flag));
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t d_tmem = tmem_base + buf * TM_BN;
-      int kb = 0;
-      // two k-blocks per trip round the loop: both stages are awaited, then one fence, eight
-      // MMAs, and the commit of each stage right after its own four
-      for (; kb + 1 < KB; kb += 2, it += 2) {
-        const uint32_t s0 = it % TM_NS, ph0 = (it / TM_NS) & 1u;
-        const uint32_t s1 = (it + 1) % TM_NS, ph1 = ((it + 1) / TM_NS) & 1u;
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[s0]), ph0, abort_flag) &&
-                                         mbar_wait(smem_u32(&bars.full[s1]), ph1, abort_flag));
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      TileM t;
+      decode_tile_m(s_meta, args, item, Nt, unit, t);
+      const bool full_item = t.rows_valid > kTileRows;
+      const uint32_t a0 = full_item ? 0u : (nh & 1u);  // accumulator of the first (or only) 128 rows
+      const uint32_t d0 = tmem_base + a0 * TM_BN;
+      for (int kb = 0; kb < KB; ++kb) {
+        bool ready = mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag);
+        // the accumulators must have been read out of tensor memory before they are overwritten
+        if (kb == 0) {
+          ready = ready && mbar_wait(smem_u32(&bars.tmem_empty[a0]), ((a0 ? n1 : n0) & 1u) ^ 1u, abort_flag);
+          if (full_item) ready = ready && mbar_wait(smem_u32(&bars.tmem_empty[1]), (n1 & 1u) ^ 1u, abort_flag);
+        }
+        ok = __all_sync(0xffffffffu, ready);
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          const uint32_t sa0 = smem_base + s0 * TM_STAGE, sa1 = smem_base + s1 * TM_STAGE;
-          const uint64_t adesc0 = smem_desc_k128(sa0), bdesc0 = smem_desc_k128(sa0 + TM_A_BYTES);
-          const uint64_t adesc1 = smem_desc_k128(sa1), bdesc1 = smem_desc_k128(sa1 + TM_A_BYTES);
-#pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)
-            umma_bf16(d_tmem, adesc0 + 2 * k, bdesc0 + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-          umma_commit(smem_u32(&bars.empty[s0]));
-#pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)
-            umma_bf16(d_tmem, adesc1 + 2 * k, bdesc1 + 2 * k, idesc, 1u);
-          umma_commit(smem_u32(&bars.empty[s1]));
-          if (kb + 2 == KB) umma_commit(smem_u32(&bars.tmem_full[buf]));
+          const uint32_t sa = smem_base + s * stage_bytes;
+          const uint64_t bdesc = smem_desc_k128(sa + b_off);
+          const uint64_t adesc0 = smem_desc_k128(sa);
+          const uint32_t acc_flag = kb > 0 ? 1u : 0u;
+          umma_bf16(d0, adesc0, bdesc, idesc, acc_flag);
+          if (owed_bar) umma_commit(owed_bar);
+          umma_bf16(d0, adesc0 + 2, bdesc + 2, idesc, 1u);
+          umma_bf16(d0, adesc0 + 4, bdesc + 4, idesc, 1u);
+          umma_bf16(d0, adesc0 + 6, bdesc + 6, idesc, 1u);
+          if (kb == KB - 1) umma_commit(smem_u32(&bars.tmem_full[a0]));  // these rows can be read already
+          if (full_item) {
+            const uint64_t adesc1 = smem_desc_k128(sa + TM_A_HALF);
+            umma_bf16(tmem_base + TM_BN, adesc1, bdesc, idesc, acc_flag);
+            umma_bf16(tmem_base + TM_BN, adesc1 + 2, bdesc + 2, idesc, 1u);
+            umma_bf16(tmem_base + TM_BN, adesc1 + 4, bdesc + 4, idesc, 1u);
+            umma_bf16(tmem_base + TM_BN, adesc1 + 6, bdesc + 6, idesc, 1u);
+            if (kb == KB - 1) umma_commit(smem_u32(&bars.tmem_full[1]));
+          }
         }
+        owed_bar = smem_u32(&bars.empty[s]);
+        if (++s == ns) { s = 0; ph ^= 1u; }
         __syncwarp();
       }
-      if (!ok) break;
-      for (; kb < KB; ++kb, ++it) {
-        const uint32_t s = it % TM_NS, ph = (it / TM_NS) & 1u;
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
-        if (lane == 0) {
-          const uint32_t sa = smem_base + s * TM_STAGE;
-          const uint64_t adesc = smem_desc_k128(sa);
-          const uint64_t bdesc = smem_desc_k128(sa + TM_A_BYTES);
-#pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)
-            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-          umma_commit(smem_u32(&bars.empty[s]));
-          if (kb == KB - 1) umma_commit(smem_u32(&bars.tmem_full[buf]));
-        }
-        __syncwarp();
-      }
+      if (full_item) { ++n0; ++n1; }
+      else { if (a0) ++n1; else ++n0; ++nh; }
     }
+    if (ok && owed_bar && lane == 0) umma_commit(owed_bar);
+    __syncwarp();
   } else {
-    // ---- epilogue (warps 2..5): warp w may touch tensor-memory lanes 32*(w%4) .. +31
+    // ---- epilogue: warp w may touch tensor-memory lanes 32 (w % 4) .. + 31.  The first half of
+    // the epilogue warps reads accumulator 0, the second half accumulator 1; where an accumulator
+    // has eight warps, the first four take the first 128 columns and the other four the rest.
+    const int e = warp - 2;
+    const uint32_t acc = (uint32_t)(e / (TM_EPI_WARPS / 2));
+    const int half = (e / 4) % (TM_EPI_WARPS / 8);   // which share of the 8 column chunks
+    constexpr int kChunks = 64 / TM_EPI_WARPS;        // 32-column chunks per warp (4 or 8)
     const int wq = warp & 3;
     const int row = 32 * wq + lane;
-    uint32_t tile_it = 0;
+    uint32_t n = 0, nh = 0;  // uses of this warp's accumulator so far; half items so far
     bool ok = true;
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile_it) {
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
       TileM t;
-      decode_tile_m(s_meta, args, item, Nt, t);
-      const uint32_t buf = tile_it & 1u, bph = (tile_it >> 1) & 1u;
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_full[buf]), bph, abort_flag));
+      decode_tile_m(s_meta, args, item, Nt, unit, t);
+      const bool full_item = t.rows_valid > kTileRows;
+      int row_half = (int)acc;  // a full item: accumulator a holds rows 128 a ..
+      if (!full_item) {
+        const uint32_t a0 = nh & 1u;
+        ++nh;
+        if (a0 != acc) continue;  // the other accumulator's item
+        row_half = 0;
+      }
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_full[acc]), n & 1u, abort_flag));
       if (!ok) break;
+      ++n;
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(32 * wq) << 16) + buf * TM_BN;
-      store_tile_tokens_m<GATE_UP, OUT>(taddr, args, t.nt, t.c, t.out_row, t.rows_valid, row);
+      const uint32_t taddr = tmem_base + ((uint32_t)(32 * wq) << 16) + acc * TM_BN;
+      store_tile_tokens_m<GATE_UP, OUT>(taddr, args, t.nt, t.c, t.out_row + row_half * kTileRows,
+                                        t.rows_valid - row_half * kTileRows, row, kChunks * half,
+                                        kChunks * (half + 1));
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[buf]));
+      if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[acc]));
     }
   }
   // the dependents may be scheduled once every CTA is this far: a grid that waits on an SM for the
   // whole run of this kernel costs issue slots and power
   pdl_launch_dependents();
-  teardown<TM_NS, 512>(bars, tmem_base, issued, args.status);
+  teardown<512>(bars, tmem_base, issued, ns, args.status);
 }
 
 // ----------------------------------------------------------------------- gemm_weights_m
@@ -840,7 +913,7 @@ gemm_weights_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args
     }
   }
   pdl_launch_dependents();
-  teardown<WM_NS, 256>(bars, tmem_base, issued, args.status);
+  teardown<256>(bars, tmem_base, issued, WM_NS, args.status);
 }
 
 // ----------------------------------------------------------------------- gemm_tokens_d
@@ -1069,7 +1142,7 @@ gemm_tokens_d_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args,
     }
   }
   pdl_launch_dependents();
-  teardown<TD_NS, 512>(bars, tmem_base, issued, args.status);
+  teardown<512>(bars, tmem_base, issued, TD_NS, args.status);
 }
 
 // ------------------------------------------------------------------ wait-expiry test hook
@@ -1102,7 +1175,7 @@ wait_expiry_kernel(int* status, unsigned long long limit_ns) {
   } else {
     (void)__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_full[0]), 0u, abort_flag, 2 * limit_ns));
   }
-  teardown<1, 32>(bars, tmem_base, 0u, status);
+  teardown<32>(bars, tmem_base, 0u, 1u, status);
 }
 
 // ------------------------------------------------------------ CUDA-core debug kernels
@@ -1241,16 +1314,24 @@ cudaError_t launch_wait_expiry(int* status, unsigned long long limit_ns, cudaStr
 }
 
 cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps& maps,
-                                 const GemmArgs& a, cudaStream_t st) {
+                                 const GemmArgs& args, cudaStream_t st) {
   const int grid = g_num_sms > 0 ? g_num_sms : 148;
+  // Items of 256 token rows move a third fewer bytes per FLOP, but a launch needs enough of them:
+  // with fewer than four rounds of items the last, partly filled round costs more than the bytes
+  // save (2048 tokens, down projection: 320 items on 148 CTAs took 0.59 ms against 0.46 ms as 576
+  // single row tiles), and such a launch runs on single row tiles.
+  GemmArgs a = args;
+  const long long Nt = (a.n_w_rows + TM_BN - 1) / TM_BN;
+  const long long items256 = ((long long)(a.est_rows + 2 * kTileRows - 1) / (2 * kTileRows) + (a.r + 1) / 2) * Nt;
+  a.single_row_tiles = items256 < 4ll * grid ? 1 : 0;
   // Plain stream order for these long kernels: launched as programmatic dependents they measured
   // 3-5 % slower at T = 8192 (5.35 vs 5.0-5.1 ms per step), while the short kernels around them and
   // the weight-major kernels gain from the overlap.
   if (gate_up)
-    return launch_plain(gemm_tokens_m_kernel<true, kOutActBf16>, dim3(grid), dim3(kThreads), TM_SMEM, st, maps, a);
+    return launch_plain(gemm_tokens_m_kernel<true, kOutActBf16>, dim3(grid), dim3(TmCfg<true>::kThreads), TM_SMEM, st, maps, a);
   if (out_kind == kOutF32)
-    return launch_plain(gemm_tokens_m_kernel<false, kOutF32>, dim3(grid), dim3(kThreads), TM_SMEM, st, maps, a);
-  return launch_plain(gemm_tokens_m_kernel<false, kOutBf16>, dim3(grid), dim3(kThreads), TM_SMEM, st, maps, a);
+    return launch_plain(gemm_tokens_m_kernel<false, kOutF32>, dim3(grid), dim3(TmCfg<false>::kThreads), TM_SMEM, st, maps, a);
+  return launch_plain(gemm_tokens_m_kernel<false, kOutBf16>, dim3(grid), dim3(TmCfg<false>::kThreads), TM_SMEM, st, maps, a);
 }
 
 cudaError_t launch_gemm_tokens_d(bool gate_up, const GemmMaps& maps, const GemmArgs& a, int kb_per_item,
