@@ -469,8 +469,8 @@ def search_case(layer, x, steps, warmup, stream, dev, rank, local, world, peaks,
     K = E if dense else E - 4 + 2
     gu_ms, dn_ms, en_ms = (stage_ms[i] / n_search for i in (1, 2, 3))
     gu_flop, dn_flop = 4 * T * K * H * F, 2 * T * K * H * F
-    # the enumeration for r reads the E - r + 2 top-ranked expert outputs of every token once
-    en_bytes = T * H * 2 * ((E - 6 + 2) + (E - 4 + 2)) + 2 * T * E * 4
+    # one enumeration pass for both sizes reads the K evaluated expert outputs of every token once
+    en_bytes = T * H * 2 * K + T * E * 4
     ach = gu_flop / (gu_ms * 1e-3) / 1e12
     step_tf = (gu_flop + dn_flop) / (ms_step * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "gemm_tokens_m_kernel<gate_up> (expert evaluations of the search)",
