@@ -841,32 +841,12 @@ def run_stack(a):
     def step():
         binding.stack_forward(layers, x, betas, 1e-5, y)
 
-    def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
-        torch.cuda.synchronize(dev)
-
-    with torch.cuda.stream(stream):
-        for _ in range(max(a.warmup, 3)):
-            step()
-    barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    with torch.cuda.stream(stream):
-        ev0.record(stream)
-        for _ in range(a.steps):
-            step()
-        ev1.record(stream)
-    barrier()
-    ms_total = ev0.elapsed_time(ev1)
-    clocks = sampler.stop() if rank == 0 else None
-    ms_total = max_over_ranks(ms_total, dev)
-    ms_step = ms_total / a.steps
-    value = whole_job_value(T, a.steps, ms_total, world)
+    barrier = make_barrier(world, dev)
+    blocks, clocks = timed_blocks(step, a.steps, a.warmup, stream, dev, rank, local, world, a.target_seconds,
+                                  max_s=30.0, min_repeats=min(MIN_REPEATS, 10))
+    timing = timing_record(blocks, a.steps, clocks)
+    ms_step = timing["ms_per_step_median"]
+    value = whole_job_value(T, 1, ms_step, world)
 
     xh = x.cpu().pin_memory()
     yh = torch.empty_like(xh).pin_memory()
@@ -918,7 +898,8 @@ def run_stack(a):
                        "final_state_rel_error_vs_unpruned": drift,
                        "parallelism": "replicas x%d, no collective" % world,
                        "l2": "each layer streams its own weights (GBs), far above the 126 MB L2"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": per_layer * NL * a.steps,
+            "timing": timing, "clocks": clocks, "e2e": e2e,
+            "gpu_launches": per_layer * NL * a.steps * timing["repeats"],
             "roofline": roofline, "cpu_baseline": None, "stages": None,
         }
         print(json.dumps(line), flush=True)
