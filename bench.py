@@ -747,13 +747,12 @@ def run_stack(a):
     # instead of searching again: the pruned layers are then built straight from the masks
     from paper_2402_14800_b200 import pruning_io
     pmeta = {"E": E, "r": r, "n_layers": NL, "h": H, "f": F, "calibration_tokens": a.cal_tokens,
-             "search_mode": a.search_mode if r < 8 else "none", "beta": a.beta, "weight_seed0": 100,
-             "calibration_seed": 1001}
-    pfile = a.pruning_file or "pruning_stack%d_%s_%s_%s_cal%d.json" % (NL, a.kept, a.search_mode, a.beta, a.cal_tokens)
+             "search_mode": a.search_mode if r < 8 else "none", "weight_seed0": 100, "calibration_seed": 1001}
+    pfile = a.pruning_file or "pruning_stack%d_%s_%s_cal%d.json" % (NL, a.kept, a.search_mode, a.cal_tokens)
     loaded = None
     if r < 8 and os.path.exists(pfile) and not a.research:
         loaded = pruning_io.load_pruning(pfile, expect_meta=pmeta)
-    all_losses = []
+    all_losses, cal_betas = [], []
     state_p = state.clone() if (r < 8 and a.search_mode == "progressive" and loaded is None) else None
     if loaded is not None:
         for l in range(NL):
@@ -763,7 +762,7 @@ def run_stack(a):
                 layer.share_scratch(layers[0])
             layers.append(layer)
             masks.append(loaded[l]["kept_mask"])
-            betas.append(loaded[l]["beta"])
+            betas.append(loaded[l]["beta"] if a.beta == "calibrated" else 0.0)
             del W
     for l in range(NL if loaded is None else 0):
         W = synth.make_layer_weights(H, F, E, seed=100 + l, device=dev)
@@ -800,13 +799,14 @@ def run_stack(a):
                 layer.share_scratch(layers[0])
             if state_p is not None:
                 state_p = layer.forward(xn_cal, 0.0, residual=state_p)
-        betas.append(layer.calibrate_beta(xn_cal) if a.beta == "calibrated" else 0.0)
+        cal_betas.append(layer.calibrate_beta(xn_cal))   # stored with the masks whatever --beta says
+        betas.append(cal_betas[-1] if a.beta == "calibrated" else 0.0)
         masks.append(mask)
         layers.append(layer)
         del W
     if r < 8 and loaded is None and rank == 0:
         pruning_io.save_pruning(pfile, pmeta, [{"kept_mask": m, "losses": ls, "beta": b}
-                                               for m, ls, b in zip(masks, all_losses, betas)])
+                                               for m, ls, b in zip(masks, all_losses, cal_betas)])
     # how far the pruned stack's calibration states ended up from the unpruned stack's
     drift = None
     if loaded is not None:
