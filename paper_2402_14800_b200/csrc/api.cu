@@ -5,6 +5,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <vector>
 
 #include "common.h"
@@ -37,11 +38,13 @@ inline int popc(uint32_t v) { return __builtin_popcount(v); }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Binomial coefficients from Pascal's triangle (n <= 16 here).
 long binom(int n, int k) {
-  if (k < 0 || k > n) return 0;
-  long r = 1;
-  for (int i = 1; i <= k; ++i) r = r * (n - k + i) / i;
-  return r;
+  if (n < 0 || k < 0 || k > n || n > 2 * kMaxE) return 0;
+  long row[2 * kMaxE + 2] = {1};
+  for (int i = 1; i <= n; ++i)
+    for (int j = i; j >= 1; --j) row[j] += row[j - 1];
+  return row[k];
 }
 
 // Test hook (moe_test_set_free_bytes_limit): an upper bound on what cudaMemGetInfo may report.
@@ -699,36 +702,47 @@ int moe_coselection(moe_layer_t* L, const void* x, int T, int32_t* counts) {
 
 uint32_t moe_frequency_subset(const int32_t* counts, int E, int r) {
   if (!counts || E < 2 || E > kMaxE || r < 1 || r > E) return 0;
-  long long freq[kMaxE];
+  // activation frequency of an expert = tokens that have it in either slot of their top-2
+  struct Entry { long long tokens; int expert; };
+  std::vector<Entry> by_use(E);
   for (int e = 0; e < E; ++e) {
-    freq[e] = 0;
-    for (int b = 0; b < E; ++b) freq[e] += (long long)counts[e * E + b] + counts[b * E + e];
+    long long row = 0, col = 0;
+    for (int o = 0; o < E; ++o) { row += counts[e * E + o]; col += counts[o * E + e]; }
+    by_use[e] = {row + col, e};
   }
+  // most used first; equal use keeps the lower expert index first
+  std::stable_sort(by_use.begin(), by_use.end(),
+                   [](const Entry& a, const Entry& b) { return a.tokens > b.tokens; });
   uint32_t mask = 0;
-  for (int k = 0; k < r; ++k) {
-    int best = -1;
-    for (int e = 0; e < E; ++e)
-      if (!((mask >> e) & 1u) && (best < 0 || freq[e] > freq[best])) best = e;
-    mask |= 1u << best;
-  }
+  for (int i = 0; i < r; ++i) mask |= 1u << by_use[i].expert;
   return mask;
 }
 
-// Subsets of r of E experts in lexicographic order of their ascending index tuples.
+// Subsets of r of E experts in lexicographic order of their ascending index tuples.  With the
+// bits of a mask read in reverse (expert 0 as the most significant bit) that order is numerically
+// descending, so the masks are produced as E-bit words with r bits set in ascending numeric order
+// (next word with the same number of bits: ripple the lowest run of ones), then reversed in
+// order and in bit position.
 static std::vector<uint32_t> subset_masks(int E, int r) {
-  std::vector<uint32_t> masks;
-  masks.reserve(binom(E, r));
-  int c[kMaxE];
-  for (int i = 0; i < r; ++i) c[i] = i;
+  std::vector<uint32_t> words;
+  words.reserve(binom(E, r));
+  const uint32_t limit = E >= 32 ? 0xffffffffu : ((1u << E) - 1u);
+  uint32_t w = (1u << r) - 1u;
   for (;;) {
+    words.push_back(w);
+    const uint32_t lowest = w & (0u - w);
+    const uint32_t ripple = w + lowest;
+    if (ripple > limit || ripple == 0) break;
+    w = ripple | (((w ^ ripple) >> 2) / lowest);
+    if (w > limit) break;
+  }
+  std::vector<uint32_t> masks(words.size());
+  for (size_t i = 0; i < words.size(); ++i) {
+    const uint32_t rev_word = words[words.size() - 1 - i];
     uint32_t m = 0;
-    for (int i = 0; i < r; ++i) m |= 1u << c[i];
-    masks.push_back(m);
-    int i = r - 1;
-    while (i >= 0 && c[i] == E - r + i) --i;
-    if (i < 0) break;
-    ++c[i];
-    for (int j = i + 1; j < r; ++j) c[j] = c[j - 1] + 1;
+    for (int b = 0; b < E; ++b)
+      if ((rev_word >> b) & 1u) m |= 1u << (E - 1 - b);
+    masks[i] = m;
   }
   return masks;
 }

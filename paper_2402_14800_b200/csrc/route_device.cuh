@@ -24,17 +24,20 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 template <int R>
 __device__ __forceinline__ void route_choose(const float (&acc)[R], int r, float beta, int& e0,
                                              int& e1, bool& skip, float& w0, float& w1, float& p1) {
-  // top-2 on the logits (softmax is increasing), ties to the lower index
+  // top-2 on the logits (softmax is increasing) in one sweep over the kept experts in index
+  // order: a logit displaces the leader or the runner-up only when strictly larger, so of equal
+  // logits the lower index ranks first
+  float l0 = acc[0], l1 = 0.f;
   e0 = 0;
-  float l0 = acc[0];
-#pragma unroll
-  for (int c = 1; c < R; ++c)
-    if (c < r && acc[c] > l0) { l0 = acc[c]; e0 = c; }
   e1 = -1;
-  float l1 = 0.f;
 #pragma unroll
-  for (int c = 0; c < R; ++c)
-    if (c < r && c != e0 && (e1 < 0 || acc[c] > l1)) { l1 = acc[c]; e1 = c; }
+  for (int c = 1; c < R; ++c) {
+    if (c < r) {
+      const float v = acc[c];
+      if (v > l0) { l1 = l0; e1 = e0; l0 = v; e0 = c; }
+      else if (e1 < 0 || v > l1) { l1 = v; e1 = c; }
+    }
+  }
   // softmax numerators relative to the maximum: p_e0 = 1, p_e1 = exp(l1 - l0); the
   // denominator cancels in the ratio, the skip test and the normalised weights
   p1 = expf(l1 - l0);

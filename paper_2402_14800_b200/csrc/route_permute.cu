@@ -534,40 +534,56 @@ router_topk_kernel(const bf16* __restrict__ x, const bf16* __restrict__ Wg, int 
     if (lane == 0) s_part[warp][c] = acc[c];
   }
   __syncthreads();
-  if (threadIdx.x != 0) return;
-  float l[kMaxE];
-  for (int c = 0; c < r; ++c) {
+  // Ranking by counting, one thread per kept expert: the rank of expert c is the number of kept
+  // experts that beat it (larger logit, or equal logit and lower index), so the expert of rank m
+  // is the m-th choice.  The k chosen experts' softmax numerators relative to the largest,
+  // p_m = exp(l_m - l_0), then go through the three fixed-order sums of the rule, which one
+  // thread evaluates (k <= 8 values).
+  __shared__ float s_l[kMaxE];
+  __shared__ float s_p[kMaxE];
+  __shared__ int s_sel[kMaxE];
+  const int c = threadIdx.x;
+  if (c < r) {
     float v = 0.f;
     for (int w = 0; w < 8; ++w) v += s_part[w][c];
-    l[c] = v;
+    s_l[c] = v;
     if (logits) logits[(size_t)t * r + c] = v;
   }
-  int sel[kMaxE];
-  float p[kMaxE];
-  unsigned left = (1u << r) - 1u;
-  for (int m = 0; m < k; ++m) {
-    int best = -1;
-    for (int c = 0; c < r; ++c)
-      if (((left >> c) & 1u) && (best < 0 || l[c] > l[best])) best = c;
-    sel[m] = best;
-    left &= ~(1u << best);
-    p[m] = expf(l[best] - l[sel[0]]);
+  __syncthreads();
+  if (c < r) {
+    const float mine = s_l[c];
+    int rank = 0;
+    for (int d = 0; d < r; ++d) {
+      const float o = s_l[d];
+      rank += (o > mine) || (o == mine && d < c);
+    }
+    if (rank < k) s_sel[rank] = c;
   }
-  float total = 0.f;
-  for (int m = 0; m < k; ++m) total += p[m];
-  float tail[kMaxE + 1];
-  tail[k] = 0.f;
-  for (int m = k - 1; m >= 1; --m) tail[m] = tail[m + 1] + p[m];
-  int istar = k;
-  for (int i = 1; i <= k; ++i)
-    if (tail[i] <= beta * total) { istar = i; break; }
-  float keep = 0.f;
-  for (int m = 0; m < istar; ++m) keep += p[m];
+  __syncthreads();
+  if (c < k) s_p[c] = expf(s_l[s_sel[c]] - s_l[s_sel[0]]);
+  __syncthreads();
+  if (c != 0) return;
+  // i* = the smallest i in 1..k whose dropped mass p_i + .. + p_{k-1} (added from the smallest
+  // value upwards) is at most beta times the whole mass p_0 + .. + p_{k-1} (added in rank order)
+  float whole = 0.f;
+  for (int m = 0; m < k; ++m) whole += s_p[m];
+  const float bound = beta * whole;
+  int istar = 1;
+  {
+    float dropped = 0.f;   // mass beyond rank i - 1, for i = k, k - 1, ..: walk down while it fits
+    int i = k;
+    while (i > 1 && dropped + s_p[i - 1] <= bound) { dropped += s_p[i - 1]; --i; }
+    // dropped = p_i + .. + p_{k-1} fits; p_{i-1} + dropped does not (or i = 1)
+    istar = i;
+  }
+  float kept_mass = 0.f;
+  for (int m = 0; m < istar; ++m) kept_mass += s_p[m];
   for (int m = 0; m < k; ++m) {
-    const float w = m < istar ? p[m] / keep : 0.f;
-    idx[(size_t)t * k + m] = sel[m];
+    const float w = m < istar ? s_p[m] / kept_mass : 0.f;
+    const int e = s_sel[m];
+    idx[(size_t)t * k + m] = e;
     wn[(size_t)t * k + m] = w;
-    if (u_idx) u_idx[(size_t)t * k + m] = kept.id[sel[m]];
+    if (u_idx) u_idx[(size_t)t * k + m] = kept.id[e];
     if (u_wn) u_wn[(size_t)t * k + m] = w;
   }
   nact[t] = istar;

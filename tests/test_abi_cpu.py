@@ -80,3 +80,23 @@ def test_null_handle_is_an_error(lib):
 def test_binding_fails_loudly_without_the_library(tmp_path):
     with pytest.raises(binding.MoeError):
         binding.load_library(str(tmp_path / "libmoe.so"))
+
+
+def test_frequency_subset_on_the_host(lib):
+    # the activation-frequency baseline: the r most used experts (row + column sums of the
+    # co-selection map), equal use resolved towards the lower index; host code, no device
+    import numpy as np
+    rng = np.random.default_rng(5)
+    for E, r in ((8, 6), (8, 4), (16, 9), (4, 2), (5, 5)):
+        counts = rng.integers(0, 50, size=(E, E)).astype(np.int32)
+        np.fill_diagonal(counts, 0)
+        if E == 8:
+            counts[3, :] = counts[5, :]      # make two experts tie
+            counts[:, 3] = counts[:, 5]
+            counts[3, 5] = counts[5, 3] = 7
+        freq = counts.sum(0).astype(np.int64) + counts.sum(1)
+        order = sorted(range(E), key=lambda e: (-int(freq[e]), e))
+        want = sum(1 << e for e in order[:r])
+        buf = (ctypes.c_int32 * (E * E))(*[int(v) for v in counts.ravel()])
+        assert lib.moe_frequency_subset(buf, E, r) == want
+    assert lib.moe_frequency_subset(None, 8, 4) == 0
