@@ -429,3 +429,32 @@ def test_top2_distance(setup, T, kept):
     layer.close()
     ok = ~tie
     np.testing.assert_allclose(got[ok], want[ok], rtol=5e-3)
+
+
+@pytest.mark.parametrize("eps", [0.25, 0.03])
+def test_prune_search_with_nearly_identical_experts(setup, eps):
+    # Experts that differ from one another by a small perturbation of common weights: every
+    # subset's loss is then a small difference of large, nearly equal expert outputs, which is
+    # where a careless evaluation of the squared errors would lose its digits.  Both the
+    # layer-wise and the progressive form must still match the oracle to the usual tolerance.
+    W = synth.make_layer_weights(H, F, E, seed=0)
+    g = torch.Generator().manual_seed(123)
+    def near(Wt):
+        base = Wt[0:1].float()
+        noise = torch.randn(Wt.shape, generator=g) * synth.WEIGHT_STD
+        return (base + eps * noise).to(torch.bfloat16).contiguous()
+    W1, W3, W2 = near(W.W1), near(W.W3), near(W.W2)
+    b = synth.bf16_bits
+    T = 300
+    x = synth.make_tokens(T, H, seed=9)
+    layer = binding.MoeLayer(W.W_gate.to(DEV), W1.to(DEV), W3.to(DEV), W2.to(DEV))
+    for r in (6, 4):
+        ora = O.prune_search_allexperts(b(x), b(W.W_gate), b(W1), b(W3), b(W2), r)
+        losses, best = layer.prune_search(x.to(DEV), r)
+        P.check_search(losses, best, ora)
+    xu = synth.make_tokens(T, H, seed=10)
+    F_ref = layer.forward(xu.to(DEV), 0.0).float().contiguous()
+    ora = O.prune_search_progressive(b(x), b(W.W_gate), b(W1), b(W3), b(W2), F_ref.cpu().numpy(), 6)
+    losses, best = layer.prune_search_progressive(x.to(DEV), F_ref, 6)
+    P.check_search(losses, best, ora)
+    layer.close()
