@@ -28,7 +28,10 @@ def _worker(rank, world, port, out):
     got = bench.max_over_ranks(ms)
     dist.barrier()
     value = bench.whole_job_value(128, 4, got, world)
-    out[rank] = (got, value, bench.dist_env()[:2])
+    # per-block times: the element-wise max over ranks, and the record built from them
+    blocks = bench.max_over_ranks_vec([10.0 + rank, 12.0 - rank, 11.0])
+    rec = bench.timing_record(blocks, 4, {"sm_mhz": 1500.0})
+    out[rank] = (got, value, bench.dist_env()[:2], blocks, rec)
     dist.destroy_process_group()
 
 
@@ -42,6 +45,10 @@ def test_max_over_ranks_and_whole_job_value_gloo():
     # two replicas of 128 tokens x 4 steps over the slower rank's 15 ms
     assert abs(res[0][1] - 2 * 128 * 4 / 15e-3) < 1e-6 and res[0][1] == res[1][1]
     assert res[0][2] == (0, 2) and res[1][2] == (1, 2)
+    assert res[0][3] == res[1][3] == [11.0, 12.0, 11.0]
+    rec = res[0][4]
+    assert rec["repeats"] == 3 and rec["ms_per_step_median"] == 11.0 / 4 and rec["ms_per_step_best"] == 11.0 / 4
+    assert abs(rec["sm_cycles_per_step_median"] - 11.0 / 4 * 1e-3 * 1500e6) < 1e-3
 
 
 def test_single_process_is_identity():
@@ -49,6 +56,7 @@ def test_single_process_is_identity():
     import bench
     assert bench.max_over_ranks(3.5) == 3.5
     assert bench.whole_job_value(10, 2, 1000.0, 1) == 20.0
+    assert bench.max_over_ranks_vec([1.0, 2.5]) == [1.0, 2.5]
 
 
 def test_reference_arm_non_zero_rank_exits_without_work():
