@@ -47,14 +47,14 @@ def measured_peaks():
     return dict(hbm=6650.0, tf_burst=1590.0, tf_sust=1400.0, source="fallback")
 
 
-def kernel_source_sha256(kernel: str):
-    """Hash of the source text of one __global__ kernel in csrc/gemm_sm100.cu (from its name to
-    the closing brace in column 0)."""
+def kernel_source_sha256(kernel: str = ""):
+    """Hash of the source file of the grouped GEMMs with its shared header: any edit to either
+    (kernel bodies, tile decoding, epilogues, descriptors) voids the recorded counters."""
     import hashlib
-    src = open(os.path.join(ROOT, "paper_2402_14800_b200", "csrc", "gemm_sm100.cu")).read()
-    i = src.index("\n" + kernel + "(")
-    j = src.index("\n}\n", i)
-    return hashlib.sha256(src[i:j].encode()).hexdigest()
+    hsh = hashlib.sha256()
+    for name in ("gemm_sm100.cu", "common.h"):
+        hsh.update(open(os.path.join(ROOT, "paper_2402_14800_b200", "csrc", name), "rb").read())
+    return hsh.hexdigest()
 
 
 def single_token_gemv() -> bool:
@@ -67,7 +67,7 @@ def single_token_gemv() -> bool:
 def recorded_traffic(workload: str, kernel: str):
     """DRAM bytes per launch of the dominant kernel from the committed ncu capture of this
     workload, or None when there is none, it is of another kernel than the one that ran, or
-    that kernel's source changed since."""
+    the GEMM sources changed since."""
     try:
         rec = json.load(open(os.path.join(ROOT, "profiles", "traffic.json"))).get(workload)
         if (rec and rec["kernel"] == kernel
