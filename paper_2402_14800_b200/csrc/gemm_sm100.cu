@@ -3,14 +3,16 @@
 //
 //   E_e(x) = W2_e ( silu(W1_e x) * (W3_e x) )      (Sec. 3.1; Mixtral's SwiGLU form)
 //
-// Two persistent, warp-specialised kernels share one pipeline skeleton:
-//   gemm_tokens_m   128 token rows x 256 weight rows per tile; for large batches, where the
-//                   work is a dense contraction bound by the tensor pipe.
+// Three persistent, warp-specialised kernels share one pipeline skeleton:
+//   gemm_tokens_m   256 token rows x 256 weight rows per item on two accumulators; for large
+//                   batches, where the work is a dense contraction bound by the tensor pipe.
 //   gemm_weights_m  128 weight rows x (16..128) tokens per item; for small batches, where
 //                   every weight byte is streamed from HBM exactly once.
-// Warp 0 issues TMA loads, warp 1 issues the MMAs (one lane) and owns the tensor memory,
-// warps 2-5 run the epilogue out of tensor memory while the next tile accumulates in the
-// other half of it.
+//   gemm_tokens_d   up to 128 token rows x 256 weight rows per item; small batches with many
+//                   tokens per expert (twice the weight bytes per trip round the MMA loop).
+// Warp 0 issues TMA loads, warp 1 issues the MMAs (one lane) and owns the tensor memory, the
+// other warps run the epilogue out of tensor memory (in the small-batch kernels while the next
+// item accumulates in the other half of it).
 //
 // W1/W3 are stored interleaved (16 gate rows, 16 up rows, ...) so that one accumulator tile
 // holds both halves of a SwiGLU feature and the epilogue can fuse silu(g) * u.
