@@ -458,3 +458,25 @@ def test_prune_search_with_nearly_identical_experts(setup, eps):
     losses, best = layer.prune_search_progressive(x.to(DEV), F_ref, 6)
     P.check_search(losses, best, ora)
     layer.close()
+
+
+@pytest.mark.parametrize("kept,beta", [(FULL, 0.3), (0b01101101, 0.0)])
+def test_forward_many_tokens_on_double_row_items(setup, kept, beta):
+    # enough tokens for the large-batch GEMM to run on items of 256 token rows at this small shape
+    # (2f = 896 weight rows: the last 256-row weight tile is half empty; ragged expert groups end
+    # in half items and partly filled tiles)
+    host, dev = setup
+    r = run_case(host, dev, 20000, kept, beta, x_seed=21)
+    assert r["ties"] <= 20000 // 20
+
+
+def test_prune_search_many_tokens_on_double_row_items(setup):
+    host, dev = setup
+    T = 9000   # two chunks of expert evaluations, the first one of 8192 tokens x 6 experts
+    x = synth.make_tokens(T, H, seed=22)
+    layer = make_layer(dev)
+    (l6, b6), (l4, b4) = layer.prune_search_multi(x.to(DEV), [6, 4])
+    layer.close()
+    xb = synth.bf16_bits(x)
+    P.check_search(l6, b6, O.prune_search_allexperts(xb, host["Wg"], host["W1"], host["W3"], host["W2"], 6))
+    P.check_search(l4, b4, O.prune_search_allexperts(xb, host["Wg"], host["W1"], host["W3"], host["W2"], 4))
