@@ -34,6 +34,7 @@ int fail(int code, const char* fmt, ...) {
   } while (0)
 
 constexpr int kMaxTokens = 1 << 24;  // per call; keeps every row index and byte count in range
+constexpr long kMaxSubsetsPerPass = 16384;  // subsets of several sizes share an enumeration pass up to here
 inline int popc(uint32_t v) { return __builtin_popcount(v); }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -775,8 +776,21 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
   const int Tc = T < 8192 ? T : 8192;  // tokens per chunk of expert evaluations
   const int Tc_pad = (int)align_up((size_t)Tc, kTileRows);
   const int nchunks = (T + Tc - 1) / Tc;
-  // per-block partial losses of the enumeration
-  const size_t partial_floats = (size_t)enumerate_num_blocks(T, (int)nC) * (size_t)nC;
+  // per-block partial losses of an enumeration pass (a pass takes at most kMaxSubsetsPerPass
+  // subsets, or one whole size if that alone is more)
+  size_t partial_floats = 0;
+  {
+    long pass = 0;
+    for (int i = 0; i <= n_r; ++i) {
+      const long n = i < n_r ? binom(E, rs[i]) : 0;
+      if (i == n_r || (pass > 0 && pass + n > kMaxSubsetsPerPass)) {
+        const size_t need = (size_t)enumerate_num_blocks(T, (int)pass) * (size_t)pass;
+        if (need > partial_floats) partial_floats = need;
+        pass = 0;
+      }
+      pass += n;
+    }
+  }
   // A subset of r experts always contains two of a token's K = E - r + 2 top-ranked experts,
   // so only those K need to be evaluated per token (all of them when K = E).
   const int K = E - r + 2;
@@ -907,18 +921,27 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
   // through one pass that reads each token's K expert outputs once; every loss is computed by
   // the same operations in the same order as in a pass of its own size.
   std::vector<std::vector<uint32_t>> masks(n_r);
-  std::vector<uint32_t> all_masks;
-  for (int i = 0; i < n_r; ++i) {
-    masks[i] = subset_masks(E, rs[i]);
-    all_masks.insert(all_masks.end(), masks[i].begin(), masks[i].end());
-  }
-  const size_t n_all = all_masks.size();
-  CUDA_TRY(cudaMemcpyAsync(W.s_subsets.p, all_masks.data(), n_all * 4, cudaMemcpyHostToDevice, st));
-  CUDA_TRY(launch_enumerate((const float*)W.s_logits.p, (const bf16*)W.s_yall.p, T, E, r, h,
-                            (const uint32_t*)W.s_subsets.p, (int)n_all, (float*)W.s_partial.p,
-                            (double*)W.s_loss_sq.p, (float*)W.s_losses.p, F_ref, src, st));
-  CUDA_TRY(cudaMemcpyAsync(losses, L->ws->s_losses.p, n_all * 4, cudaMemcpyDeviceToHost, st));
+  for (int i = 0; i < n_r; ++i) masks[i] = subset_masks(E, rs[i]);
   size_t o = 0;
+  for (int i0 = 0; i0 < n_r;) {
+    // sizes i0 .. i1 - 1 go through one pass (as many as the per-warp loss table has room for)
+    std::vector<uint32_t> batch = masks[i0];
+    int i1 = i0 + 1;
+    while (i1 < n_r && batch.size() + masks[i1].size() <= (size_t)kMaxSubsetsPerPass) {
+      batch.insert(batch.end(), masks[i1].begin(), masks[i1].end());
+      ++i1;
+    }
+    const size_t n = batch.size();
+    CUDA_TRY(cudaMemcpyAsync(W.s_subsets.p, batch.data(), n * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(launch_enumerate((const float*)W.s_logits.p, (const bf16*)W.s_yall.p, T, E, r, h,
+                              (const uint32_t*)W.s_subsets.p, (int)n, (float*)W.s_partial.p,
+                              (double*)W.s_loss_sq.p, (float*)W.s_losses.p, F_ref, src, st));
+    CUDA_TRY(cudaMemcpyAsync(losses + o, L->ws->s_losses.p, n * 4, cudaMemcpyDeviceToHost, st));
+    // the host list is reused for the next pass: the copy above must have left it
+    if (i1 < n_r) CUDA_TRY(cudaStreamSynchronize(st));
+    o += n;
+    i0 = i1;
+  }
   mark(L);
   if ((rc = check_status(L))) return rc;
   o = 0;

@@ -480,3 +480,26 @@ def test_prune_search_many_tokens_on_double_row_items(setup):
     xb = synth.bf16_bits(x)
     P.check_search(l6, b6, O.prune_search_allexperts(xb, host["Wg"], host["W1"], host["W3"], host["W2"], 6))
     P.check_search(l4, b4, O.prune_search_allexperts(xb, host["Wg"], host["W1"], host["W3"], host["W2"], 4))
+
+
+def test_prune_search_multi_in_several_passes():
+    # 16 experts: the subsets of sizes 15, 14 and 8 (13006 together) share one enumeration pass, the
+    # 11440 of size 7 need a second one; every size must give what a search of its own gives (to
+    # rounding: with more than six ranked experts per token the errors are formed pair by pair)
+    build.build()
+    E_, h, f, T = 16, 128, 192, 150
+    W = synth.make_layer_weights(h, f, E_, seed=61)
+    x = synth.make_tokens(T, h, seed=62).to(DEV)
+    layer = binding.MoeLayer(W.W_gate.to(DEV), W.W1.to(DEV), W.W3.to(DEV), W.W2.to(DEV))
+    rs = [15, 14, 8, 7]
+    multi = layer.prune_search_multi(x, rs)
+    for r, (losses, best) in zip(rs, multi):
+        single, best1 = layer.prune_search(x, r)
+        assert len(losses) == len(single) == binding.num_subsets(E_, r)
+        np.testing.assert_allclose(losses, single, rtol=2e-5, atol=1e-7)
+        if best != best1:
+            assert abs(min(losses) - single[int(np.argmin(losses))]) <= 1e-4 * min(single)
+    b = synth.bf16_bits
+    ora = O.prune_search_allexperts(b(x), b(W.W_gate), b(W.W1), b(W.W3), b(W.W2), 14)
+    P.check_search(multi[1][0], multi[1][1], ora)
+    layer.close()
