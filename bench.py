@@ -581,6 +581,82 @@ def matrix_rows(W, xcal, layers, stream, dev, rank, local, world, peaks, head):
     return rows
 
 
+def stack_matrix_rows(stream, dev, rank, local, world, peaks, n_layers=32, T=16, cal_tokens=4096):
+    """Two rows of the 32-layer stack (x <- x + MoE_l(RMSNorm(x)), a seed per layer, attention left
+    out) at decode size: all experts kept, and pruned to r = 4 with each layer's subset from the
+    layer-wise search on calibration states of the unpruned stack (searched while the unpruned
+    stack is built).  The stacks are built one after the other: 90 GB, then 45 GB of weights."""
+    from paper_2402_14800_b200 import binding
+    x = synth.make_tokens(T, H, seed=1, device=dev)
+    y = torch.empty_like(x)
+    rows = []
+
+    def time_stack(layers, name, masks, extra):
+        for l in layers:
+            l.set_stream(stream)
+        betas = [0.0] * len(layers)
+        touched = []
+        with torch.cuda.stream(stream):
+            cur = x
+            stats = binding.RoutingStats(T, E, dev)
+            for layer in layers:
+                cur = layer.forward(binding.rmsnorm(cur, stream=stream), 0.0, residual=cur, stats=stats)
+                stream.synchronize()
+                touched.append(int(stats.n_experts_touched.item()))
+        blocks, clocks = timed_blocks(lambda: binding.stack_forward(layers, x, betas, 1e-5, y), 3, 3, stream, dev,
+                                      rank, local, world, target_s=1.0, max_s=5.0, min_repeats=10)
+        tr = timing_record(blocks, 3, clocks)
+        ms = tr["ms_per_step_median"]
+        nbytes = sum(touched) * 3 * H * F * 2
+        row = {"workload": name, "tokens": T, "layers": len(layers), "tokens_per_s": T / (ms * 1e-3),
+               "ms_per_step": ms, "ms_per_step_best": tr["ms_per_step_best"], "repeats": tr["repeats"],
+               "steps_per_block": 3, "weight_bytes": sum(l.weight_bytes for l in layers),
+               "experts_touched_sum": sum(touched), "bound": "hbm", "unit": "GB/s",
+               "algorithmic_bytes": nbytes, "whole_step_frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm"],
+               "peak": peaks["hbm"], "kept_masks": masks, "clocks": clocks}
+        row.update(extra)
+        return row
+
+    # pass 1: the unpruned stack; every layer is searched for r = 4 on the way
+    state = synth.make_tokens(cal_tokens, H, seed=1001, device=dev)
+    layers, masks4, search_s = [], [], 0.0
+    for l in range(n_layers):
+        W = synth.make_layer_weights(H, F, E, seed=100 + l, device=dev)
+        layer = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, 0xFF)
+        del W
+        if layers:
+            layer.share_scratch(layers[0])
+        xn = binding.rmsnorm(state)
+        torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        masks4.append(layer.prune_search(xn, 4)[1])
+        search_s += time.perf_counter() - t0
+        state = layer.forward(xn, 0.0, residual=state)
+        layers.append(layer)
+    del state, xn
+    rows.append(time_stack(layers, "stack%d_T%d_full_beta-0" % (n_layers, T), [0xFF] * n_layers, {}))
+    for layer in reversed(layers):
+        layer.close()
+    layers = []
+    torch.cuda.empty_cache()
+    # pass 2: the stack pruned to the searched subsets
+    for l in range(n_layers):
+        W = synth.make_layer_weights(H, F, E, seed=100 + l, device=dev)
+        layer = binding.MoeLayer(W.W_gate, W.W1, W.W3, W.W2, masks4[l])
+        del W
+        if layers:
+            layer.share_scratch(layers[0])
+        layers.append(layer)
+    rows.append(time_stack(layers, "stack%d_T%d_r4_beta-0" % (n_layers, T), masks4,
+                           {"search_wall_s_all_layers": search_s, "calibration_tokens": cal_tokens,
+                            "speedup_vs_unpruned_beta0": rows[0]["ms_per_step"] / 1.0}))
+    rows[1]["speedup_vs_unpruned_beta0"] = rows[0]["ms_per_step"] / rows[1]["ms_per_step"]
+    for layer in reversed(layers):
+        layer.close()
+    torch.cuda.empty_cache()
+    return rows
+
+
 def run_ours(a):
     from paper_2402_14800_b200 import binding, build
     rank, world, local = dist_env()
@@ -689,6 +765,11 @@ def run_ours(a):
         for k, l in layers.items():
             if l is not layer:
                 l.close()
+        if a.stack_rows:
+            del W
+            torch.cuda.empty_cache()
+            matrix += stack_matrix_rows(stream, dev, rank, local, world, peaks)
+            W = None
         matrix_s = time.perf_counter() - t0
 
     if rank == 0:
@@ -935,6 +1016,8 @@ def main():
                     help="headline workload only (the default decode run also measures the other configured workloads)")
     ap.add_argument("--min-repeats", type=int, default=30,
                     help="blocks of --steps steps in the timed region at least (1 with --target-seconds 0 for a profiler)")
+    ap.add_argument("--no-stack-rows", dest="stack_rows", action="store_false",
+                    help="leave the two 32-layer stack rows (90 GB + 45 GB of weights) out of the matrix")
     ap.add_argument("--target-seconds", type=float, default=1.5,
                     help="device time the repeated blocks of the timed region should cover")
     a = ap.parse_args()
