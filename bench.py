@@ -494,13 +494,13 @@ def search_case(layer, x, steps, warmup, stream, dev, rank, local, world, peaks,
                 launches_per_step=chunks * 7 + 2 * 2)
 
 
-def matrix_rows(W, xcal, layers, stream, dev, rank, local, world, peaks, head):
+def matrix_rows(W, xcal, layers, stream, dev, rank, local, world, peaks, head, rows):
     """The other configured workloads, measured in the same invocation after the headline: decode
     at T = 1 / 8 / 32 and on pruned layers, prefill at T = 2048 / 8192 / 32768 with skipping off
     and on, the pruning search at T = 32768.  Each row has its own timed blocks, clock record and
     roofline fractions; speed-ups are against the same kernels on the unpruned layer at beta = 0."""
     from paper_2402_14800_b200 import binding
-    rows, base_ms = [], {}
+    base_ms = {}   # `rows` is the caller's list: what has been measured survives a failure later on
 
     def layer_for(kname):
         if kname not in layers:
@@ -764,7 +764,7 @@ def run_ours(a):
         # the headline line must come out whatever happens in the extra rows
         matrix = []
         try:
-            matrix = matrix_rows(W, xcal, layers, stream, dev, rank, local, world, peaks, c)
+            matrix_rows(W, xcal, layers, stream, dev, rank, local, world, peaks, c, matrix)
         except Exception as e:  # noqa: BLE001
             matrix.append({"workload": "matrix", "error": repr(e)})
         for k, l in layers.items():
