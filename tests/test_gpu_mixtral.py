@@ -118,7 +118,7 @@ def test_small_batches_repeat_bit_for_bit(big, T):
 
 def test_search_subsample_matches_oracle(big):
     host = big["host"]
-    x = synth.make_tokens(40, H, seed=1, device=DEV)
+    x = synth.make_tokens(96, H, seed=1, device=DEV)
     layer = big["layer"](FULL)
     for r in (6, 4):
         ora = O.prune_search_allexperts(synth.bf16_bits(x), host["Wg"], host["W1"], host["W3"], host["W2"], r)
@@ -145,6 +145,17 @@ def test_search_full_size_invariants(big):
     assert l6 == whole and b6 == best
     l4s, b4s = layer.prune_search(x, 4)
     assert l4 == l4s and b4 == b4s and len(l4) == 70
+    # the same losses through the forward path at full size: F'(x, C) and F(x) from two layer
+    # forwards (pruned handle, unpruned handle; other kernels, outputs rounded to bf16), so the two
+    # agree to the bf16 rounding of the outputs
+    y_full = layer.forward(x, 0.0).double()
+    for C in (best, int(O.enumerate_subsets(8, 6)[int(np.argmax(whole))])):
+        y_pruned = big["layer"](C).forward(x, 0.0).double()
+        loss_fw = float((y_pruned - y_full).norm())
+        loss_search = whole[list(O.enumerate_subsets(8, 6)).index(C)]
+        assert abs(loss_fw - loss_search) <= 2e-2 * loss_search, (hex(C), loss_fw, loss_search)
+        del y_pruned
+    del y_full
     # the loss of a subset is carried by the tokens whose top-2 it breaks: more broken tokens, on
     # average, more loss -- checked through the routing record of the same batch
     stats = binding.RoutingStats(T, E, DEV)
