@@ -211,6 +211,20 @@ def test_topk_and_progressive_at_full_shape(big):
     both = (idx == ora["idx"]).all(1) & (na == ora["n_active"])
     assert both.sum() >= 20
     P.check_outputs(synth.bf16_bits(y), ora["y"], both)
+    # the same at a large batch (large-batch GEMMs on three slots per token), the oracle on its
+    # first 32 tokens
+    xl = synth.make_tokens(3000, H, seed=8, device=DEV)
+    xlb = synth.bf16_bits(xl)[:32]
+    ora_l = O.moe_forward_topk(xlb, host["Wg"], host["W1"], host["W3"], host["W2"], FULL, 3, 0.2)
+    yl, idl, wnl, nal = layer.forward_topk(xl, 3, 0.2, record=True)
+    torch.cuda.synchronize()
+    idl, nal = idl.cpu().numpy()[:32], nal.cpu().numpy()[:32]
+    srt_l = -np.sort(-ora_l["logits"].astype(np.float64), axis=1)
+    tie_l = (np.diff(-srt_l[:, :4], axis=1) < P.LOGIT_GAP_TOL).any(1)
+    assert np.array_equal(idl[~tie_l], ora_l["idx"][~tie_l])
+    both_l = (idl == ora_l["idx"]).all(1) & (nal == ora_l["n_active"])
+    assert both_l.sum() >= 28
+    P.check_outputs(synth.bf16_bits(yl)[:32], ora_l["y"], both_l)
     # progressive search: target from other tokens' unpruned outputs
     xu = synth.make_tokens(24, H, seed=4, device=DEV)
     F_ref = layer.forward(xu, 0.0).float().contiguous()
