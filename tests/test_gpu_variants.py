@@ -283,3 +283,22 @@ def test_reserve_makes_later_calls_allocation_free(weights):
     with pytest.raises(binding.MoeError):
         layer.reserve(0)
     layer.close()
+
+
+@pytest.mark.parametrize("T", [1, 40, 700])
+def test_plain_stream_order_gives_the_same_bits(weights, T):
+    # MOE_NO_PDL=1: every kernel in plain stream order instead of as a programmatic dependent;
+    # the overlap of launches must not change a single bit
+    x = synth.make_tokens(T, H, seed=8).to(DEV)
+    ref = binding.MoeLayer(*weights, 0b11011101)
+    want = ref.forward(x, 0.4).clone()
+    ref.close()
+    plain = layer_with_env(weights, 0b11011101, MOE_NO_PDL=1)
+    try:
+        got = plain.forward(x, 0.4).clone()
+        torch.cuda.synchronize()
+        assert plain.device_status() == 0
+    finally:
+        plain.close()
+        layer_with_env(weights, MOE_NO_PDL=0).close()  # the switch is process-wide: back to the default
+    assert torch.equal(got, want)
