@@ -83,7 +83,8 @@ int moe_layer_share_scratch(moe_layer_t* layer, moe_layer_t* owner);
  */
 int moe_reserve(moe_layer_t* layer, int T_max);
 
-/* Bytes of device memory the handle holds for weights (router + kept experts). */
+/* Bytes of device memory the handle holds for weights: the kept experts' three
+ * matrices and the router rows (stored padded with zero rows to 16 rows). */
 size_t moe_layer_weight_bytes(const moe_layer_t* layer);
 
 /* Bytes of device memory the handle currently holds as scratch. */

@@ -354,7 +354,13 @@ int forward_impl(moe_layer* L, const void* x, int T, float beta, const void* res
                                          (int32_t*)L->ws->pair_pos.p, (int32_t*)L->ws->row_token.p,
                                          (bf16*)L->ws->xperm.p, s_count, s_nsk, s_nt, L->kept, L->E, st));
   } else {
-    CUDA_TRY(launch_router((const bf16*)x, L->Wg, T, L->h, L->r, beta, L->kept, ro, st));
+    // the tensor-core router wins from about 64 tiles of 128 tokens on (T = 8192: routing stage
+    // 0.144 -> 0.115 ms, T = 32768: 0.52 -> 0.35 ms; T = 4096 equal, T = 2048 slower on its 16 CTAs)
+    if (L->debug_simt || T < 64 * kTileRows)
+      CUDA_TRY(launch_router((const bf16*)x, L->Wg, T, L->h, L->r, beta, L->kept, ro, st));
+    else
+      CUDA_TRY(launch_router_tc((const bf16*)x, L->Wg, T, L->h, L->r, beta, L->kept, ro,
+                                (int*)L->ws->status.p, st));
     CUDA_TRY(launch_scan(ro.blk_hist, nblk, L->r, kTileRows, (int32_t*)L->ws->blk_base.p, meta,
                          s_count, s_nsk, s_nt, L->kept, L->E, st));
     CUDA_TRY(cudaMemsetAsync(L->ws->row_token.p, 0xff, (size_t)rows_cap * 4, st));
@@ -469,7 +475,8 @@ moe_layer_t* moe_layer_create(const void* W_gate, const void* W1, const void* W3
   const char* dense = getenv("MOE_SEARCH_DENSE");
   L->search_dense = dense && dense[0] == '1';
 
-  const size_t n_gate = (size_t)L->r * h * 2, n_13 = (size_t)L->r * 2 * f * h * 2,
+  // the router rows are padded with zero rows to kMaxE rows (the tensor-core router's operand)
+  const size_t n_gate = (size_t)kMaxE * h * 2, n_13 = (size_t)L->r * 2 * f * h * 2,
                n_2 = (size_t)L->r * h * f * 2;
   size_t free_b = 0;
   if (free_device_bytes(&free_b) != cudaSuccess) free_b = ~(size_t)0;
@@ -488,6 +495,7 @@ moe_layer_t* moe_layer_create(const void* W_gate, const void* W1, const void* W3
     return nullptr;
   }
   L->weight_bytes = n_gate + n_13 + n_2;
+  ok = cudaMemsetAsync(L->Wg, 0, n_gate, 0) == cudaSuccess;
   for (int c = 0; c < L->r && ok; ++c) {
     const int id = L->kept.id[c];
     ok = ok && cudaMemcpyAsync(L->Wg + (size_t)c * h, (const bf16*)W_gate + (size_t)id * h,

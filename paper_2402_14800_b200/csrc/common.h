@@ -123,6 +123,10 @@ struct RouteOut {
 
 cudaError_t launch_router(const bf16* x, const bf16* Wg, int T, int h, int r, float beta,
                           const KeptIds& kept, const RouteOut& out, cudaStream_t st);
+// Large batches (T > kDecodeMaxT): the logits on the tensor cores (gemm_sm100.cu), the decision as
+// in launch_router.  Wg16 = the kept router rows padded with zero rows to kMaxE rows.
+cudaError_t launch_router_tc(const bf16* x, const bf16* Wg16, int T, int h, int r, float beta,
+                             const KeptIds& kept, const RouteOut& out, int* status, cudaStream_t st);
 // T <= kDecodeMaxT: router with one block per token; permutation + gather with one block per token
 cudaError_t launch_router_small(const bf16* x, const bf16* Wg, int T, int h, int r, float beta,
                                 const KeptIds& kept, const RouteOut& out, cudaStream_t st);

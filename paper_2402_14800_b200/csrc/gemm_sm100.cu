@@ -23,6 +23,7 @@
 #include <stdio.h>
 
 #include "common.h"
+#include "route_device.cuh"
 
 namespace moe {
 
@@ -1147,6 +1148,169 @@ gemm_tokens_d_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args,
   teardown<512>(bars, tmem_base, issued, TD_NS, args.status);
 }
 
+// -------------------------------------------------------------------- router_tc (large T)
+//
+// Router logits of a large batch on the tensor cores (Sec. 3.1: l = W_gate x over the kept
+// experts): a [T x h] x [h x 16] contraction that has to read every token row once and nothing
+// else, so it runs at the rate the rows arrive.  One CTA takes tiles of 128 tokens in turn: the
+// producer warp streams the tile's k-blocks (128 rows x 64 values, 16 KB) and the matching
+// k-blocks of the 16 padded router rows (2 KB) through an 8-stage ring, one lane issues four
+// M128 N16 K16 MMAs per k-block.
+// The tensor core does not round its fp32 accumulation the IEEE way, and over a whole row of
+// 4096 products with outlier channels that left the logits accurate to 5e-5 only.  So the
+// accumulator holds no more than kRouterChunkKb k-blocks (128 products) at a time: the MMA lane
+// alternates between two 16-column accumulators, one chunk each, and the four epilogue warps, one
+// thread per token, read every chunk out of tensor memory and add it to the token's logits with
+// IEEE fp32 additions in chunk order.  The routing decision (top-2, skip test, weights:
+// route_decide) is then taken exactly as the CUDA-core routers take it.  Each epilogue warp also
+// writes the pair counts of its two blocks of 16 tokens, the histogram rows the permutation's
+// scan reads.
+
+constexpr int RT_NS = 8;
+constexpr int RT_X_BYTES = 128 * 128;   // 128 token rows x 64 bf16
+constexpr int RT_W_BYTES = 16 * 128;    // 16 router rows x 64 bf16
+constexpr int RT_STAGE = RT_X_BYTES + RT_W_BYTES;
+constexpr int RT_SMEM = RT_NS * RT_STAGE + 1024;
+constexpr int RT_N = 16;                // accumulator columns = padded router rows
+constexpr int kRouterChunkKb = 2;       // k-blocks accumulated inside the tensor core at a time
+
+struct RouterMaps {
+  CUtensorMap x;   // token rows [T][h], box 64 x 128
+  CUtensorMap wg;  // router rows [16][h] (rows beyond the kept experts are zero), box 64 x 16
+};
+
+template <int R>
+__global__ void __launch_bounds__(kThreads, 1)
+router_tc_kernel(const __grid_constant__ RouterMaps maps, int T, int h, int r, float beta, KeptIds kept,
+                 RouteOut o, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ Bars bars;
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  setup_barriers<RT_NS>(bars);
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars.tmem_base), 32);
+    tmem_relinquish();
+  }
+  pdl_launch_dependents();
+  pdl_wait();  // the token rows may have been written by the stream's previous kernel
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *(volatile uint32_t*)&bars.tmem_base;
+  volatile int* abort_flag = &bars.abort_flag;
+  const int KB = (h + BK - 1) / BK;
+  const int n_chunks = (KB + kRouterChunkKb - 1) / kRouterChunkKb;
+  const int n_tiles = (T + 127) / 128;
+  uint32_t issued = 0;
+
+  if (warp == 0) {
+    uint32_t it = 0, s = 0, ph = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int kb = 0; kb < KB; ++kb, ++it) {
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag));
+        if (!ok) break;
+        if (lane == 0) {
+          const uint32_t full = smem_u32(&bars.full[s]);
+          const uint32_t sa = smem_base + s * RT_STAGE;
+          mbar_expect_tx(full, RT_STAGE);
+          tma_load_2d(sa, &maps.x, kb * BK, tile * 128, full);
+          tma_load_2d(sa + RT_X_BYTES, &maps.wg, kb * BK, 0, full);
+        }
+        if (++s == RT_NS) { s = 0; ph ^= 1u; }
+        __syncwarp();
+      }
+    }
+    issued = it;
+  } else if (warp == 1) {
+    const uint32_t idesc = idesc_bf16(128, RT_N);
+    uint32_t s = 0, ph = 0, chunk_it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int kb = 0; kb < KB; ++kb) {
+        const bool first = kb % kRouterChunkKb == 0;
+        const bool last = kb % kRouterChunkKb == kRouterChunkKb - 1 || kb == KB - 1;
+        const uint32_t buf = chunk_it & 1u, bph = (chunk_it >> 1) & 1u;
+        bool ready = mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag);
+        if (first) ready = ready && mbar_wait(smem_u32(&bars.tmem_empty[buf]), bph ^ 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ready);
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t sa = smem_base + s * RT_STAGE;
+          const uint64_t adesc = smem_desc_k128(sa);
+          const uint64_t bdesc = smem_desc_k128(sa + RT_X_BYTES);
+          const uint32_t d_tmem = tmem_base + buf * RT_N;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
+          umma_commit(smem_u32(&bars.empty[s]));
+          if (last) umma_commit(smem_u32(&bars.tmem_full[buf]));
+        }
+        if (last) ++chunk_it;
+        if (++s == RT_NS) { s = 0; ph ^= 1u; }
+        __syncwarp();
+      }
+    }
+  } else {
+    // epilogue warp wq owns tensor-memory lanes 32 wq .. 32 wq + 31 = tokens 32 wq .. of the tile
+    const int wq = warp & 3;
+    uint32_t chunk_it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      float acc[R], lost[R];  // compensated (Kahan) sums of the chunks: `lost` carries what an addition dropped
+#pragma unroll
+      for (int c = 0; c < R; ++c) { acc[c] = 0.f; lost[c] = 0.f; }
+      for (int ch = 0; ch < n_chunks; ++ch, ++chunk_it) {
+        const uint32_t buf = chunk_it & 1u, bph = (chunk_it >> 1) & 1u;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tmem_full[buf]), bph, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t v[16];
+        tmem_ld16(tmem_base + ((uint32_t)(32 * wq) << 16) + buf * RT_N, v);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars.tmem_empty[buf]));
+#pragma unroll
+        for (int c = 0; c < R; ++c) {
+          const float term = __fsub_rn(__uint_as_float(v[c]), lost[c]);
+          const float sum = __fadd_rn(acc[c], term);
+          lost[c] = __fsub_rn(__fsub_rn(sum, acc[c]), term);
+          acc[c] = sum;
+        }
+      }
+      if (!ok) break;
+      const int t = tile * 128 + 32 * wq + lane;
+      int e0 = -1, e1 = -1;
+      bool skip = false;
+      if (t < T) {
+        route_decide<R>(acc, r, beta, t, kept, o, e0, e1, skip);
+        if (skip) e1 = -1;
+      }
+      if (o.blk_hist) {
+        // pair counts of the two blocks of kRouteTokPerBlock = 16 tokens this warp holds
+        const int blk = (tile * 128 + 32 * wq) / kRouteTokPerBlock;
+        const int nblk = (T + kRouteTokPerBlock - 1) / kRouteTokPerBlock;
+#pragma unroll 1
+        for (int col = 0; col < kHistCols; ++col) {
+          bool hit;
+          if (col == 2 * kMaxE) hit = skip;
+          else hit = ((col & 1) ? e1 : e0) == (col >> 1);
+          const unsigned m = __ballot_sync(0xffffffffu, hit);
+          if (lane == 0) {
+            if (blk < nblk) o.blk_hist[(size_t)blk * kHistCols + col] = __popc(m & 0xffffu);
+            if (blk + 1 < nblk) o.blk_hist[(size_t)(blk + 1) * kHistCols + col] = __popc(m >> 16);
+          }
+        }
+      }
+    }
+  }
+  teardown<32>(bars, tmem_base, issued, RT_NS, status);
+}
+
 // ------------------------------------------------------------------ wait-expiry test hook
 
 // One CTA with the GEMMs' barrier block and a tensor-memory allocation.  Warp 0 waits, with the
@@ -1301,6 +1465,11 @@ cudaError_t gemm_set_attributes() {
   SET_ATTR((gemm_weights_m_kernel<false, 64>), WmCfg<64>::kSmem)
   SET_ATTR((gemm_weights_m_kernel<true, 128>), WmCfg<128>::kSmem)
   SET_ATTR((gemm_weights_m_kernel<false, 128>), WmCfg<128>::kSmem)
+  SET_ATTR((router_tc_kernel<2>), RT_SMEM)
+  SET_ATTR((router_tc_kernel<4>), RT_SMEM)
+  SET_ATTR((router_tc_kernel<6>), RT_SMEM)
+  SET_ATTR((router_tc_kernel<8>), RT_SMEM)
+  SET_ATTR((router_tc_kernel<kMaxE>), RT_SMEM)
   SET_ATTR((gemm_tokens_d_kernel<true>), TD_SMEM)
   SET_ATTR((gemm_tokens_d_kernel<false>), TD_SMEM)
 #undef SET_ATTR
@@ -1308,6 +1477,27 @@ cudaError_t gemm_set_attributes() {
   e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   return cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+}
+
+cudaError_t launch_router_tc(const bf16* x, const bf16* Wg16, int T, int h, int r, float beta,
+                             const KeptIds& kept, const RouteOut& out, int* status, cudaStream_t st) {
+  RouterMaps maps;
+  if (make_map_2d(&maps.x, x, (uint64_t)h, (uint64_t)T, 128) || make_map_2d(&maps.wg, Wg16, (uint64_t)h, kMaxE, RT_N))
+    return cudaErrorInvalidValue;
+  const int n_tiles = (T + 127) / 128;
+  int grid = g_num_sms > 0 ? g_num_sms : 148;
+  if (grid > n_tiles) grid = n_tiles;
+#define MOE_ROUTER_TC(R)                                                                          \
+  return launch_pdl(router_tc_kernel<R>, dim3(grid), dim3(kThreads), RT_SMEM, st, maps, T, h, r, beta, kept, \
+                    out, status)
+  switch (r) {
+    case 2: MOE_ROUTER_TC(2);
+    case 3: case 4: MOE_ROUTER_TC(4);
+    case 5: case 6: MOE_ROUTER_TC(6);
+    case 7: case 8: MOE_ROUTER_TC(8);
+    default: MOE_ROUTER_TC(kMaxE);
+  }
+#undef MOE_ROUTER_TC
 }
 
 cudaError_t launch_wait_expiry(int* status, unsigned long long limit_ns, cudaStream_t st) {
