@@ -159,6 +159,17 @@ def workload_name(a):
     return "%s_T%d_%s_beta-%s" % (a.workload, a.tokens, a.kept, a.beta)
 
 
+def layer_config(a, T, kept_mask, beta, pairs, touched, world):
+    """The `config` object of a single-layer line; both arms build it here so that the two lines
+    name the same workload with the same keys."""
+    return {"workload": workload_name(a), "h": H, "f": F, "E": E, "tokens": T,
+            "kept_mask": kept_mask, "beta": beta, "pairs": pairs, "experts_touched": touched,
+            "parallelism": "replicas x%d, no collective" % world,
+            "l2": "per step the kernels stream %.2f GB of weights, far above the 126 MB L2"
+                  % (touched * 3 * H * F * 2 / 1e9) if a.workload != "search" else
+                  "inputs and intermediates are GBs, far above the 126 MB L2"}
+
+
 # ------------------------------------------------------------------------- reference arm
 
 def oracle_sample(a, W_host, x_host, beta, n_sample):
@@ -262,12 +273,22 @@ def run_reference(a):
     value = n_sample * per_unit * a.steps / sum(times)
     metric, unit = metric_unit(a)
     sample = "%d of %d tokens per step, oracle as it stands" % (n_sample, a.tokens)
+    # the workload's pair and expert counts, from the oracle's own routing of the whole batch
+    kept_mask = KEPT[a.kept]
+    if a.workload == "search":
+        pairs = touched = 0
+    else:
+        rt = O.route(xh, Wh["Wg"], kept_mask, beta)
+        alive = np.ones_like(rt["idx"], dtype=bool)
+        alive[:, 1] = rt["skipped"] == 0
+        pairs = int(alive.sum())
+        touched = int(len(np.unique(rt["idx"][alive])))
     line = {
         "impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": a.gpus,
         "steps": a.steps, "warmup": a.warmup, "ms_per_step": 1e3 * sum(times) / a.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": workload_name(a), "h": H, "f": F, "E": E, "beta": beta},
+        "config": layer_config(a, a.tokens, kept_mask, beta, pairs, touched, max(a.gpus, 1)),
         "cpu_baseline": {"value": value, "unit": unit, "cores": O.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -786,12 +807,7 @@ def run_ours(a):
             "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": a.steps,
             "warmup": max(a.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": workload_name(a), "h": H, "f": F, "E": E, "tokens": T,
-                       "kept_mask": kept, "beta": beta, "pairs": pairs, "experts_touched": touched,
-                       "parallelism": "replicas x%d, no collective" % world,
-                       "l2": "per step the kernels stream %.2f GB of weights, far above the 126 MB L2"
-                             % (touched * 3 * H * F * 2 / 1e9) if a.workload != "search" else
-                             "inputs and intermediates are GBs, far above the 126 MB L2"},
+            "config": layer_config(a, T, kept, beta, pairs, touched, world),
             "timing": timing, "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches_per_step * a.steps * timing["repeats"],
             "gpu_launches_per_step": launches_per_step, "roofline": roofline,
