@@ -266,10 +266,8 @@ int check_status(moe_layer* L) {
 // The two grouped GEMMs of the experts over a batch described by `meta`.
 int run_expert_gemms(moe_layer* L, const Meta* meta, bool weights_m, const GemmMaps& m_gu,
                      const GemmMaps& m_dn, GemmArgs gu, GemmArgs dn, GemmOut dn_kind,
-                     const bf16* gu_A, const bf16* dn_A, int simt_rows, int T = 0, int est_rows = 0) {
+                     const bf16* gu_A, const bf16* dn_A, int simt_rows, int T = 0) {
   gu.meta = meta; dn.meta = meta;
-  // rows of the batch at most (by default the capacity in rows, which bounds the pairs that run)
-  gu.est_rows = dn.est_rows = est_rows > 0 ? est_rows : simt_rows;
   gu.r = L->r; dn.r = L->r;
   gu.K = L->h; gu.n_w_rows = 2 * L->f;
   dn.K = L->f; dn.n_w_rows = L->h;
@@ -913,7 +911,7 @@ static int search_impl(moe_layer_t* L, const void* x_calib, const float* F_ref, 
       dn.a_off_mul = 1; dn.out_row_base = t0; dn.out_off_mul = 0; dn.out_col_mul = h;
       dn.out_ld = (long long)E * h; dn.out = W.s_yall.p;
       if ((rc = run_expert_gemms(L, meta, false, m_gu, m_dn, gu, dn, kOutBf16, xa,
-                                 (const bf16*)W.s_act.p, rows, 0, E * rows))) {
+                                 (const bf16*)W.s_act.p, rows))) {
         L->prof = prof_saved;
         return rc;
       }

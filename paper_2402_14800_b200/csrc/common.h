@@ -193,8 +193,6 @@ struct GemmArgs {
   void* out;               // bf16 activations / fp32 outputs / bf16 expert outputs
   long long split_stride;  // elements between split-K partial planes (decode down-proj)
   int* status;             // device error word
-  int est_rows;            // token-expert pairs of the batch at most (sizes the items of the large-batch kernel)
-  int single_row_tiles;    // large-batch kernel: items of one 128-row tile instead of two (set by its launcher)
   // weight-major kernel: arrival counters (kTailHeaderBytes, zero between launches) followed by
   // the partial tiles of the K-sliced tail items; null = no slicing
   float* tail;

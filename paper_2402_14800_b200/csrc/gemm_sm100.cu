@@ -308,7 +308,7 @@ template <bool GATE_UP> struct TmCfg {
 };
 
 // An item covers `unit` row tiles of 128 (2 normally; 1 for launches with too few items to fill
-// the machine with double row tiles, see launch_gemm_tokens_m).  Items of expert c:
+// the machine with double row tiles: the kernel decides, see below).  Items of expert c:
 // ceil(row tiles / unit) x Nt weight tiles, ordered band of kBand / unit row items -> weight
 // tile -> row item, so that the items in flight share few token tiles and weight tiles in L2.
 __device__ __forceinline__ void decode_tile_m(const Meta& m, const GemmArgs& a, int item, int Nt,
@@ -420,9 +420,17 @@ gemm_tokens_m_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs args)
 
   const int KB = (args.K + BK - 1) / BK;
   const int Nt = (args.n_w_rows + TM_BN - 1) / TM_BN;
-  // single row tiles per item: 4 stages of 48 KB (one token tile + the weight tile), every item
-  // a half item; the accumulators then alternate, which double-buffers them
-  const bool single = args.single_row_tiles != 0;
+  // Items of 256 token rows move a third fewer bytes per FLOP, but a launch needs enough of them:
+  // an item of one row tile (4 stages of 48 KB: one token tile + the weight tile; every item a
+  // half item, the accumulators alternate, which double-buffers them) takes about 0.58 of a
+  // double-row item's time, and the last, partly filled round of a launch costs a whole item.
+  // Every CTA compares the rounds of both forms from the real group sizes (2048 tokens, down
+  // projection: 3 rounds of double-row items 0.55 ms, 4 rounds of single-row items 0.50 ms;
+  // 3072 tokens: 3 rounds 0.60 ms against 6 rounds 0.72 ms).
+  const int grid = (int)gridDim.x;
+  const int rounds1 = (num_items_m(s_meta, args, Nt, 1) + grid - 1) / grid;
+  const int rounds2 = (num_items_m(s_meta, args, Nt, 2) + grid - 1) / grid;
+  const bool single = 58 * rounds1 < 100 * rounds2;
   const int unit = single ? 1 : 2;
   const uint32_t ns = single ? 4u : (uint32_t)TM_NS;
   const uint32_t stage_bytes = single ? (uint32_t)(TM_A_HALF + TM_B_BYTES) : (uint32_t)TM_STAGE;
@@ -1508,14 +1516,7 @@ cudaError_t launch_wait_expiry(int* status, unsigned long long limit_ns, cudaStr
 cudaError_t launch_gemm_tokens_m(bool gate_up, GemmOut out_kind, const GemmMaps& maps,
                                  const GemmArgs& args, cudaStream_t st) {
   const int grid = g_num_sms > 0 ? g_num_sms : 148;
-  // Items of 256 token rows move a third fewer bytes per FLOP, but a launch needs enough of them:
-  // with fewer than four rounds of items the last, partly filled round costs more than the bytes
-  // save (2048 tokens, down projection: 320 items on 148 CTAs took 0.59 ms against 0.46 ms as 576
-  // single row tiles), and such a launch runs on single row tiles.
-  GemmArgs a = args;
-  const long long Nt = (a.n_w_rows + TM_BN - 1) / TM_BN;
-  const long long items256 = ((long long)(a.est_rows + 2 * kTileRows - 1) / (2 * kTileRows) + (a.r + 1) / 2) * Nt;
-  a.single_row_tiles = items256 < 4ll * grid ? 1 : 0;
+  const GemmArgs& a = args;
   // Plain stream order for these long kernels: launched as programmatic dependents they measured
   // 3-5 % slower at T = 8192 (5.35 vs 5.0-5.1 ms per step), while the short kernels around them and
   // the weight-major kernels gain from the overlap.
