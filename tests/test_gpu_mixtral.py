@@ -75,8 +75,8 @@ def test_decode_batches(big, T, mode):
     run_case(big, T, FULL, beta)
 
 
-@pytest.mark.parametrize("T,mode", [(2048, "beta0"), (2048, "calibrated"), (8192, "beta0"), (8192, "calibrated"),
-                                     (32768, "beta0"), (32768, "calibrated")])
+@pytest.mark.parametrize("T,mode", [(512, "beta0"), (2048, "beta0"), (2048, "calibrated"), (3072, "calibrated"),
+                                     (8192, "beta0"), (8192, "calibrated"), (32768, "beta0"), (32768, "calibrated")])
 def test_prefill_batches(big, T, mode):
     beta = 0.0 if mode == "beta0" else calibrated_beta(big, FULL)
     worst, sk = run_case(big, T, FULL, beta)
